@@ -1,0 +1,112 @@
+/*
+ * attn.h -- C ABI of the B200 (sm_100a) fused attention forward library.
+ *
+ * The operation is the one the paper states in Section 2.2 ("Attention computation"):
+ *
+ *     O = softmax(Q K^T * scale [+ causal mask]) V
+ *
+ * evaluated tile by tile with a running row maximum and row sum (the FlashAttention
+ * scheme the same section describes), for multi-head attention (Section 4.2) and
+ * grouped-query attention (Section 4.3), BF16 inputs, head dimension 128
+ * (Section 4.1, "Benchmark Configurations").  In addition the library returns the
+ * per-row log-sum-exp of the scaled visible scores, which the paper does not mention.
+ *
+ * Everything is `extern "C"`, plain pointers and integers.  No entry point throws,
+ * aborts or prints; each returns an attn_status_t.
+ */
+#ifndef ATTN_B200_ATTN_H_
+#define ATTN_B200_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ATTN_OK = 0,
+  ATTN_ERR_NULL = 1,        /* a required pointer is NULL */
+  ATTN_ERR_SHAPE = 2,       /* a dimension is <= 0, or Hq is not a multiple of Hkv */
+  ATTN_ERR_UNSUPPORTED = 3, /* D != 128; causal with Sq > Sk; scale not finite or < 0 */
+  ATTN_ERR_ALIGN = 4,       /* q, k, v or o not 16-byte aligned; lse not 4-byte aligned */
+  ATTN_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed (descriptor, launch, copy) */
+  ATTN_ERR_ARCH = 6,        /* the current device is not compute capability 10.x */
+  ATTN_ERR_TIMEOUT = 7      /* a bounded wait inside a kernel expired (see attn_last_device_status) */
+} attn_status_t;
+
+/*
+ * attn_fwd -- fused attention forward (Section 2.2; GQA head mapping per Section 4.3:
+ * consecutive query heads share a key/value head, hkv = hq / (Hq / Hkv)).
+ *
+ * All pointers are DEVICE pointers on the current device, owned by the caller; the
+ * library neither frees nor retains them.  The call is asynchronous: work is enqueued
+ * on `stream` and the function returns without synchronising.
+ *
+ *   q    BF16 [B, Sq, Hq,  D]  contiguous, D innermost            (read)
+ *   k    BF16 [B, Sk, Hkv, D]                                     (read)
+ *   v    BF16 [B, Sk, Hkv, D]                                     (read)
+ *   o    BF16 [B, Sq, Hq,  D]  rounded to nearest even from fp32  (written)
+ *   lse  FP32 [B, Hq, Sq]      natural-log sum of exp(scale * q.k_j) over the visible
+ *                              keys of each row; may be NULL to skip   (written)
+ *   B, Hq, Hkv, Sq, Sk  any positive sizes (lengths need not be multiples of the
+ *                       128-row tile); Hq % Hkv == 0
+ *   D        must be 128
+ *   causal   0: every key is visible.  non-zero: key j is visible to query i iff
+ *            j <= i + (Sk - Sq)  (lower-triangular when Sq == Sk); requires Sq <= Sk
+ *   scale    multiplies Q K^T; finite and >= 0 (callers normally pass 1/sqrt(D))
+ *   stream   cudaStream_t (NULL = default stream)
+ *
+ * o must not alias q, k or v.  Distinct streams may call concurrently.  The first
+ * call on a device allocates a few KB of library-owned device state (tile-scheduler
+ * counters and a status word); tensors are never allocated.
+ * Arithmetic: S and O accumulate in fp32 on the tensor cores; P = exp2 of the scaled,
+ * max-subtracted scores is rounded to BF16 before P V; the row sum is taken in fp32
+ * before that rounding.
+ */
+attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+                       int B, int Hq, int Hkv, int Sq, int Sk, int D,
+                       int causal, float scale, void* stream);
+
+/*
+ * attn_fwd_host -- the same operation on HOST buffers (same layouts).  Copies q, k, v
+ * to library-owned device staging buffers (grown on demand, kept for later calls),
+ * runs attn_fwd, copies o and lse (if not NULL) back and synchronises `stream` before
+ * returning.  Pinned host memory makes the copies asynchronous with respect to the
+ * host; pageable memory works too.  Not re-entrant: one call at a time per process.
+ */
+attn_status_t attn_fwd_host(const void* q, const void* k, const void* v, void* o, float* lse,
+                            int B, int Hq, int Hkv, int Sq, int Sk, int D,
+                            int causal, float scale, void* stream);
+
+/* Releases the staging buffers attn_fwd_host holds on the current device. */
+attn_status_t attn_release_host_staging(void);
+
+/*
+ * attn_set_option -- tuning / A-B switches; returns ATTN_ERR_UNSUPPORTED for an
+ * unknown name or value.  Options are process-wide and read at each launch.
+ *   "scheduler"   0 = one CTA per work item (hardware block scheduler)
+ *                 1 = persistent CTAs, static round-robin over work items
+ *                 2 = persistent CTAs, dynamic work counter (default)
+ *   "max_ctas"    0 = one per SM (default), else an upper bound on persistent CTAs
+ */
+attn_status_t attn_set_option(const char* name, int value);
+
+/* Human-readable name of a status code (static storage). */
+const char* attn_status_str(attn_status_t status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int attn_version(void);
+
+/*
+ * attn_last_device_status -- synchronises the current device and reads the status word
+ * kernels write when one of their bounded waits expires.  *code is 0 when nothing
+ * expired, else identifies the waiting role; *detail identifies the barrier.  Returns
+ * ATTN_ERR_TIMEOUT when *code != 0 (the word is then cleared), ATTN_OK otherwise.
+ */
+attn_status_t attn_last_device_status(int* code, int* detail);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATTN_B200_ATTN_H_ */

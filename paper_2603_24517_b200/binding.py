@@ -1,0 +1,147 @@
+"""ctypes binding of the C ABI in ``include/attn.h`` -- argument marshalling only.
+
+Every step of the attention forward pass runs in the CUDA library; torch is used for
+device memory and streams.  The library is never substituted: if ``libattn_b200.so``
+is missing or fails to load, importing a symbol here raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libattn_b200.so")
+
+ATTN_OK = 0
+STATUS_NAMES = {
+    0: "ATTN_OK", 1: "ATTN_ERR_NULL", 2: "ATTN_ERR_SHAPE", 3: "ATTN_ERR_UNSUPPORTED", 4: "ATTN_ERR_ALIGN",
+    5: "ATTN_ERR_CUDA", 6: "ATTN_ERR_ARCH", 7: "ATTN_ERR_TIMEOUT",
+}
+EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_host", "attn_release_host_staging", "attn_set_option",
+                    "attn_status_str", "attn_version", "attn_last_device_status")
+
+_lib = None
+
+
+class AttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads ``libattn_b200.so`` (built by ``paper_2603_24517_b200.build``); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} not found: run `python -m paper_2603_24517_b200.build` "
+                          "(there is no fallback implementation)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    fwd_args = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, vp]
+    lib.attn_fwd.argtypes = fwd_args
+    lib.attn_fwd.restype = ci
+    lib.attn_fwd_host.argtypes = fwd_args
+    lib.attn_fwd_host.restype = ci
+    lib.attn_release_host_staging.argtypes = []
+    lib.attn_release_host_staging.restype = ci
+    lib.attn_set_option.argtypes = [ctypes.c_char_p, ci]
+    lib.attn_set_option.restype = ci
+    lib.attn_status_str.argtypes = [ci]
+    lib.attn_status_str.restype = ctypes.c_char_p
+    lib.attn_version.argtypes = []
+    lib.attn_version.restype = ci
+    lib.attn_last_device_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
+    lib.attn_last_device_status.restype = ci
+    _lib = lib
+    return lib
+
+
+def _check_layout(q, k, v, o, lse, device_type):
+    for name, t in (("q", q), ("k", k), ("v", v), ("o", o)):
+        if t.dtype != torch.bfloat16 or t.dim() != 4 or not t.is_contiguous() or t.device.type != device_type:
+            raise ValueError(f"{name} must be a contiguous 4-D bfloat16 {device_type} tensor [B, S, H, D]")
+    B, Sq, Hq, D = q.shape
+    Bk, Sk, Hkv, Dk = k.shape
+    if v.shape != k.shape or o.shape != q.shape or Bk != B or Dk != D:
+        raise ValueError("inconsistent q/k/v/o shapes")
+    if lse is not None:
+        if lse.dtype != torch.float32 or not lse.is_contiguous() or tuple(lse.shape) != (B, Hq, Sq) \
+                or lse.device.type != device_type:
+            raise ValueError("lse must be a contiguous float32 tensor [B, Hq, Sq]")
+    return B, Hq, Hkv, Sq, Sk, D
+
+
+def attn_fwd_status(q, k, v, o, lse, causal: bool, scale: float, stream=None) -> int:
+    """Calls ``attn_fwd`` on CUDA tensors and returns its raw status code (no exception)."""
+    B, Hq, Hkv, Sq, Sk, D = _check_layout(q, k, v, o, lse, "cuda")
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        return load_library().attn_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                       None if lse is None else lse.data_ptr(),
+                                       B, Hq, Hkv, Sq, Sk, D, int(bool(causal)), float(scale), stream)
+
+
+def attn_fwd(q, k, v, o, lse, causal: bool, scale: float, stream=None) -> None:
+    """``attn_fwd`` of the C ABI on CUDA tensors: q [B,Sq,Hq,D], k/v [B,Sk,Hkv,D] -> o, lse
+    (lse may be None).  Asynchronous on ``stream`` (default: torch's current stream)."""
+    st = attn_fwd_status(q, k, v, o, lse, causal, scale, stream)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_fwd")
+
+
+def attn_fwd_host(q, k, v, o, lse, causal: bool, scale: float, device=0, stream=None) -> None:
+    """``attn_fwd_host`` of the C ABI on CPU tensors (pinned or pageable); synchronous."""
+    B, Hq, Hkv, Sq, Sk, D = _check_layout(q, k, v, o, lse, "cpu")
+    dev = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
+    if stream is None:
+        stream = torch.cuda.current_stream(dev).cuda_stream
+    with torch.cuda.device(dev):
+        st = load_library().attn_fwd_host(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                          None if lse is None else lse.data_ptr(),
+                                          B, Hq, Hkv, Sq, Sk, D, int(bool(causal)), float(scale), stream)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_fwd_host")
+
+
+def attn_release_host_staging() -> None:
+    st = load_library().attn_release_host_staging()
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_release_host_staging")
+
+
+def attn_set_option(name: str, value: int) -> None:
+    st = load_library().attn_set_option(name.encode(), int(value))
+    if st != ATTN_OK:
+        raise AttnError(st, f"attn_set_option({name}={value})")
+
+
+def attn_status_str(status: int) -> str:
+    return load_library().attn_status_str(int(status)).decode()
+
+
+def attn_version() -> int:
+    return load_library().attn_version()
+
+
+def attn_last_device_status():
+    """(status, code, detail) -- synchronises the device."""
+    code, detail = ctypes.c_int(0), ctypes.c_int(0)
+    st = load_library().attn_last_device_status(ctypes.byref(code), ctypes.byref(detail))
+    return st, code.value, detail.value
+
+
+def attention_forward(q, k, v, causal: bool = False, scale: float | None = None, return_lse: bool = True):
+    """Convenience wrapper: allocates o (and lse) with torch and calls ``attn_fwd``."""
+    if scale is None:
+        scale = 1.0 / math.sqrt(q.shape[-1])
+    o = torch.empty_like(q)
+    lse = torch.empty((q.shape[0], q.shape[2], q.shape[1]), dtype=torch.float32, device=q.device) \
+        if return_lse else None
+    attn_fwd(q, k, v, o, lse, causal, scale)
+    return (o, lse) if return_lse else o

@@ -1,0 +1,274 @@
+// Host side of the C ABI declared in include/attn.h: argument checks, TMA descriptors,
+// persistent-grid set-up and the launch of attn_fwd_kernel.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/attn.h"
+#include "attn_fwd_kernel.cuh"
+
+namespace {
+
+using attn::FwdParams;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr int kMaxDevices = 64;
+constexpr int kCounterSlots = 1024;  // one work counter per launch in flight, reused round-robin
+
+struct DeviceState {
+  bool ready = false;
+  bool failed = false;
+  int sm_count = 0;
+  unsigned int* counters = nullptr;  // [kCounterSlots]
+  int* status = nullptr;             // [2]
+  std::atomic<unsigned int> next_slot{0};
+  // attn_fwd_host staging
+  void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  size_t stage_bytes[5] = {0, 0, 0, 0, 0};
+};
+
+std::mutex g_mutex;
+DeviceState g_dev[kMaxDevices];
+EncodeTiledFn g_encode = nullptr;
+std::atomic<int> g_opt_scheduler{2};
+std::atomic<int> g_opt_max_ctas{0};
+
+// Per-device one-time set-up: architecture check, kernel attribute, scheduler counters and
+// status word.  Returns the state or nullptr (with *st set).
+DeviceState* device_state(attn_status_t* st) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    *st = ATTN_ERR_CUDA;
+    return nullptr;
+  }
+  DeviceState& d = g_dev[dev];
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (d.ready) return &d;
+  if (d.failed) {
+    *st = ATTN_ERR_ARCH;
+    return nullptr;
+  }
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+    *st = ATTN_ERR_CUDA;
+    return nullptr;
+  }
+  if (major != 10) {
+    d.failed = true;
+    *st = ATTN_ERR_ARCH;
+    return nullptr;
+  }
+  if (g_encode == nullptr) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        fn == nullptr) {
+      *st = ATTN_ERR_CUDA;
+      return nullptr;
+    }
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaFuncSetAttribute(attn::attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           attn::kSmemBytes) != cudaSuccess ||
+      cudaMalloc(&d.counters, kCounterSlots * sizeof(unsigned int)) != cudaSuccess ||
+      cudaMalloc(&d.status, 2 * sizeof(int)) != cudaSuccess ||
+      cudaMemset(d.status, 0, 2 * sizeof(int)) != cudaSuccess) {
+    *st = ATTN_ERR_CUDA;
+    return nullptr;
+  }
+  d.ready = true;
+  return &d;
+}
+
+// [B, S, H, 128] BF16 tensor seen as 4-D (D, H, S, B); box = 64 elements x 1 head x 128 rows,
+// 128-byte swizzle, out-of-range rows read as zero and are clipped on store.
+bool make_tensor_map(CUtensorMap* tm, const void* base, int B, int S, int H) {
+  const cuuint64_t dims[4] = {128, static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(S),
+                              static_cast<cuuint64_t>(B)};
+  const cuuint64_t strides[3] = {128ull * 2, static_cast<cuuint64_t>(H) * 128 * 2,
+                                 static_cast<cuuint64_t>(S) * H * 128 * 2};
+  const cuuint32_t box[4] = {64, 1, 128, 1};
+  const cuuint32_t elem_strides[4] = {1, 1, 1, 1};
+  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+                  elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+attn_status_t check_args(const void* q, const void* k, const void* v, void* o, const float* lse, int B, int Hq,
+                         int Hkv, int Sq, int Sk, int D, int causal, float scale, bool device_ptrs) {
+  if (q == nullptr || k == nullptr || v == nullptr || o == nullptr) return ATTN_ERR_NULL;
+  if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || D <= 0) return ATTN_ERR_SHAPE;
+  if (Hq % Hkv != 0) return ATTN_ERR_SHAPE;
+  if (D != attn::kHeadDim) return ATTN_ERR_UNSUPPORTED;
+  if (causal && Sq > Sk) return ATTN_ERR_UNSUPPORTED;
+  if (!std::isfinite(scale) || !(scale > 0.f)) return ATTN_ERR_UNSUPPORTED;
+  // sizes the 32-bit tile arithmetic and the TMA coordinates can hold
+  if (static_cast<long long>(B) * Hq * ((Sq + 127) / 128) > 0x3fffffffLL) return ATTN_ERR_UNSUPPORTED;
+  if (Sq > 0x3fffff00 || Sk > 0x3fffff00) return ATTN_ERR_UNSUPPORTED;
+  if (device_ptrs) {
+    const uintptr_t mask = 15;
+    if ((reinterpret_cast<uintptr_t>(q) & mask) || (reinterpret_cast<uintptr_t>(k) & mask) ||
+        (reinterpret_cast<uintptr_t>(v) & mask) || (reinterpret_cast<uintptr_t>(o) & mask))
+      return ATTN_ERR_ALIGN;
+    if (lse != nullptr && (reinterpret_cast<uintptr_t>(lse) & 3)) return ATTN_ERR_ALIGN;
+  }
+  return ATTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
+                       int Sq, int Sk, int D, int causal, float scale, void* stream) {
+  attn_status_t st = check_args(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, scale, true);
+  if (st != ATTN_OK) return st;
+  DeviceState* dev = device_state(&st);
+  if (dev == nullptr) return st;
+
+  CUtensorMap tm_q, tm_k, tm_v, tm_o;
+  if (!make_tensor_map(&tm_q, q, B, Sq, Hq) || !make_tensor_map(&tm_k, k, B, Sk, Hkv) ||
+      !make_tensor_map(&tm_v, v, B, Sk, Hkv) || !make_tensor_map(&tm_o, o, B, Sq, Hq))
+    return ATTN_ERR_CUDA;
+
+  FwdParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
+  p.group = Hq / Hkv;
+  p.causal = causal ? 1 : 0;
+  p.off = Sk - Sq;
+  p.n_qt = (Sq + attn::kTile - 1) / attn::kTile;
+  p.n_kb = (Sk + attn::kTile - 1) / attn::kTile;
+  p.pair_heads = (p.group % 2 == 0) ? 1 : 0;
+  if (p.pair_heads) {
+    p.items_per_group = p.n_qt * (p.group / 2);
+    p.n_work = B * Hkv * p.items_per_group;
+  } else {
+    p.items_per_group = (p.n_qt + 1) / 2;
+    p.n_work = B * Hq * p.items_per_group;
+  }
+  p.scale = scale;
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.lse = lse;
+  p.status = dev->status;
+
+  const int sched = g_opt_scheduler.load();
+  int grid = p.n_work;
+  if (sched != 0) {
+    int cap = dev->sm_count;
+    const int max_ctas = g_opt_max_ctas.load();
+    if (max_ctas > 0 && max_ctas < cap) cap = max_ctas;
+    if (grid > cap) grid = cap;
+  }
+  p.dynamic = (sched == 2) ? 1 : 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (p.dynamic) {
+    const unsigned int slot = dev->next_slot.fetch_add(1) % kCounterSlots;
+    p.counter = dev->counters + slot;
+    if (cudaMemsetAsync(p.counter, 0, sizeof(unsigned int), s) != cudaSuccess) return ATTN_ERR_CUDA;
+  }
+  attn::attn_fwd_kernel<<<grid, attn::kThreads, attn::kSmemBytes, s>>>(tm_q, tm_k, tm_v, tm_o, p);
+  return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+attn_status_t attn_fwd_host(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq,
+                            int Hkv, int Sq, int Sk, int D, int causal, float scale, void* stream) {
+  attn_status_t st = check_args(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, scale, false);
+  if (st != ATTN_OK) return st;
+  DeviceState* dev = device_state(&st);
+  if (dev == nullptr) return st;
+  const size_t q_bytes = static_cast<size_t>(B) * Sq * Hq * D * 2;
+  const size_t kv_bytes = static_cast<size_t>(B) * Sk * Hkv * D * 2;
+  const size_t lse_bytes = static_cast<size_t>(B) * Hq * Sq * 4;
+  const size_t need[5] = {q_bytes, kv_bytes, kv_bytes, q_bytes, lse_bytes};
+  for (int i = 0; i < 5; ++i) {
+    if (dev->stage_bytes[i] < need[i]) {
+      if (dev->stage[i] != nullptr) cudaFree(dev->stage[i]);
+      dev->stage[i] = nullptr;
+      dev->stage_bytes[i] = 0;
+      if (cudaMalloc(&dev->stage[i], need[i]) != cudaSuccess) return ATTN_ERR_CUDA;
+      dev->stage_bytes[i] = need[i];
+    }
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(dev->stage[0], q, q_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(dev->stage[1], k, kv_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(dev->stage[2], v, kv_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return ATTN_ERR_CUDA;
+  st = attn_fwd(dev->stage[0], dev->stage[1], dev->stage[2], dev->stage[3],
+                static_cast<float*>(dev->stage[4]), B, Hq, Hkv, Sq, Sk, D, causal, scale, stream);
+  if (st != ATTN_OK) return st;
+  if (cudaMemcpyAsync(o, dev->stage[3], q_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ATTN_ERR_CUDA;
+  if (lse != nullptr &&
+      cudaMemcpyAsync(lse, dev->stage[4], lse_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return ATTN_ERR_CUDA;
+  return cudaStreamSynchronize(s) == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+attn_status_t attn_release_host_staging(void) {
+  int devid = 0;
+  if (cudaGetDevice(&devid) != cudaSuccess || devid < 0 || devid >= kMaxDevices) return ATTN_ERR_CUDA;
+  DeviceState& d = g_dev[devid];
+  for (int i = 0; i < 5; ++i) {
+    if (d.stage[i] != nullptr) cudaFree(d.stage[i]);
+    d.stage[i] = nullptr;
+    d.stage_bytes[i] = 0;
+  }
+  return ATTN_OK;
+}
+
+attn_status_t attn_set_option(const char* name, int value) {
+  if (name == nullptr) return ATTN_ERR_NULL;
+  if (std::strcmp(name, "scheduler") == 0) {
+    if (value < 0 || value > 2) return ATTN_ERR_UNSUPPORTED;
+    g_opt_scheduler.store(value);
+    return ATTN_OK;
+  }
+  if (std::strcmp(name, "max_ctas") == 0) {
+    if (value < 0) return ATTN_ERR_UNSUPPORTED;
+    g_opt_max_ctas.store(value);
+    return ATTN_OK;
+  }
+  return ATTN_ERR_UNSUPPORTED;
+}
+
+const char* attn_status_str(attn_status_t status) {
+  switch (status) {
+    case ATTN_OK: return "ATTN_OK";
+    case ATTN_ERR_NULL: return "ATTN_ERR_NULL";
+    case ATTN_ERR_SHAPE: return "ATTN_ERR_SHAPE";
+    case ATTN_ERR_UNSUPPORTED: return "ATTN_ERR_UNSUPPORTED";
+    case ATTN_ERR_ALIGN: return "ATTN_ERR_ALIGN";
+    case ATTN_ERR_CUDA: return "ATTN_ERR_CUDA";
+    case ATTN_ERR_ARCH: return "ATTN_ERR_ARCH";
+    case ATTN_ERR_TIMEOUT: return "ATTN_ERR_TIMEOUT";
+  }
+  return "ATTN_ERR_UNKNOWN";
+}
+
+int attn_version(void) { return 100; }
+
+attn_status_t attn_last_device_status(int* code, int* detail) {
+  if (code == nullptr || detail == nullptr) return ATTN_ERR_NULL;
+  attn_status_t st = ATTN_OK;
+  DeviceState* dev = device_state(&st);
+  if (dev == nullptr) return st;
+  int host[2] = {0, 0};
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(host, dev->status, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return ATTN_ERR_CUDA;
+  *code = host[0];
+  *detail = host[1];
+  if (host[0] != 0) {
+    cudaMemset(dev->status, 0, sizeof(host));
+    return ATTN_ERR_TIMEOUT;
+  }
+  return ATTN_OK;
+}
+
+}  // extern "C"

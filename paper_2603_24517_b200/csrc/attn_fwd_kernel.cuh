@@ -1,0 +1,629 @@
+// Fused attention forward for sm_100a: one persistent, warp-specialised kernel.
+//
+// Per CTA (512 threads, one CTA per SM) two 128-row query tiles ("stages") are in flight:
+//
+//   warps 0-3    softmax, stage 0   one thread per query row: S from tensor memory, online
+//   warps 4-7    softmax, stage 1   max / sum in the exp2 domain, P (BF16) back to tensor memory,
+//                                   rescale of the O accumulator when the row maximum moved
+//   warps 8-11   epilogue           O / l -> BF16 -> shared memory -> TMA store, LSE store
+//   warp  12     MMA issue          tcgen05.mma: S = Q K^T (smem x smem), O += P V (tmem x smem)
+//   warp  13     loader             TMA loads of Q tiles and of the K / V tile ring, work counter
+//   warps 14-15  idle (they only donate registers)
+//
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P aliases the first
+// 64 columns of its S.  Shared memory: Q0, Q1 (32 KB each, reused as the O staging tiles) and a
+// ring of 32 KB K / V tiles, all 128-byte swizzled [128 rows][64 elements] half tiles.
+#pragma once
+
+#include "ptx.cuh"
+
+namespace attn {
+
+constexpr int kTile = 128;        // rows per Q tile and keys per K/V tile
+constexpr int kHeadDim = 128;
+constexpr int kTileBytes = kTile * kHeadDim * 2;  // 32 KB
+constexpr int kHalfBytes = kTileBytes / 2;        // one [128][64] half tile
+constexpr int kKvSlots = 5;
+constexpr int kThreads = 512;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units a row maximum may lag behind
+
+// Registers per thread of each role after the setmaxnreg re-split of the CTA's 64K registers:
+// 8 softmax warps, 4 epilogue warps, 4 other warps; 8 * a + 4 * b + 4 * c must not exceed 2048.
+#ifndef ATTN_REGS_SOFTMAX
+#define ATTN_REGS_SOFTMAX 176
+#endif
+#ifndef ATTN_REGS_EPILOGUE
+#define ATTN_REGS_EPILOGUE 80
+#endif
+#ifndef ATTN_REGS_OTHER
+#define ATTN_REGS_OTHER 80
+#endif
+static_assert(8 * ATTN_REGS_SOFTMAX + 4 * ATTN_REGS_EPILOGUE + 4 * ATTN_REGS_OTHER <= 2048, "register split");
+
+constexpr int kSmemQ = 0;
+constexpr int kSmemKv = 2 * kTileBytes;
+constexpr int kSmemStats = kSmemKv + kKvSlots * kTileBytes;  // float [2 stages][2][128]
+constexpr int kSmemBars = kSmemStats + 2 * 2 * kTile * 4;
+constexpr int kNumBars = 2 + 2 + 2 * kKvSlots + 2 * 9;
+constexpr int kSmemMisc = kSmemBars + kNumBars * 8;  // tmem base, abort flag, sched slots
+constexpr int kSmemBytes = kSmemMisc + 32;
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every in-kernel wait gives up after 2 s
+
+struct FwdParams {
+  int B, Hq, Hkv, Sq, Sk;
+  int group;        // Hq / Hkv
+  int causal;
+  int off;          // Sk - Sq
+  int n_qt;         // ceil(Sq / 128)
+  int n_kb;         // ceil(Sk / 128)
+  int pair_heads;   // 1: the two stages hold two query heads of one KV head at the same rows
+                    // 0: the two stages hold two consecutive row tiles of one query head
+  int items_per_group;  // work items per (b, hq) [pair rows] or per (b, hkv) [pair heads]
+  int n_work;
+  int dynamic;      // 1: work items come from the global counter
+  float scale;
+  float scale_log2; // scale * log2(e)
+  float* lse;
+  unsigned int* counter;  // dynamic scheduler: next work item - gridDim.x
+  int* status;            // [0] code of the first expired wait (0 = none), [1] detail
+};
+
+struct Work {
+  int b, hkv;
+  int hq[2];
+  int row0[2];
+  int n[2];     // K/V blocks each stage visits (0 = stage unused)
+  int nmax;
+};
+
+__device__ __forceinline__ void decode_work(const FwdParams& p, int w, Work& wk) {
+  const int grp = w / p.items_per_group;
+  const int r = w - grp * p.items_per_group;
+  if (p.pair_heads) {
+    const int hp = p.group >> 1;
+    int qt = r / hp;
+    const int pp = r - qt * hp;
+    if (p.causal) qt = p.n_qt - 1 - qt;
+    wk.b = grp / p.Hkv;
+    wk.hkv = grp - wk.b * p.Hkv;
+    wk.hq[0] = wk.hkv * p.group + 2 * pp;
+    wk.hq[1] = wk.hq[0] + 1;
+    wk.row0[0] = wk.row0[1] = qt * kTile;
+  } else {
+    int qp = p.causal ? (p.items_per_group - 1 - r) : r;
+    wk.b = grp / p.Hq;
+    wk.hq[0] = wk.hq[1] = grp - wk.b * p.Hq;
+    wk.hkv = wk.hq[0] / p.group;
+    wk.row0[0] = qp * 2 * kTile;
+    wk.row0[1] = wk.row0[0] + kTile;
+  }
+#pragma unroll
+  for (int s = 0; s < 2; ++s) {
+    if (wk.row0[s] >= p.Sq) {
+      wk.n[s] = 0;
+    } else if (p.causal) {
+      const int last_row = min(wk.row0[s] + kTile, p.Sq) - 1;
+      wk.n[s] = min(p.n_kb, (last_row + p.off) / kTile + 1);
+    } else {
+      wk.n[s] = p.n_kb;
+    }
+  }
+  wk.nmax = max(wk.n[0], wk.n[1]);
+}
+
+// ------------------------------------------------------------------------------------------
+// Bounded mbarrier wait.  Returns false after kWaitLimitNs, or as soon as any thread of the
+// CTA has given up; the first to give up records (code, detail) in the global status word.
+// ------------------------------------------------------------------------------------------
+struct WaitCtx {
+  volatile int* abort_flag;  // shared memory
+  int* status;               // global
+};
+
+__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, WaitCtx ctx, int code) {
+  const uint64_t t0 = global_timer_ns();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*ctx.abort_flag) return false;
+    if (global_timer_ns() - t0 > kWaitLimitNs) {
+      *ctx.abort_flag = 1;
+      if (atomicCAS(ctx.status, 0, code) == 0) ctx.status[1] = static_cast<int>(blockIdx.x);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, WaitCtx ctx, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, ctx, code);
+}
+
+// codes: role << 8 | barrier
+enum : int {
+  kRoleLoad = 1 << 8, kRoleMma = 2 << 8, kRoleSoftmax = 3 << 8, kRoleEpilogue = 4 << 8,
+  kBarQFull = 1, kBarQEmpty = 2, kBarKvFull = 3, kBarKvEmpty = 4, kBarSFull = 5, kBarPFull = 6,
+  kBarOFull = 7, kBarOEmpty = 8, kBarLFull = 9, kBarLEmpty = 10, kBarSchedFull = 11, kBarSchedEmpty = 12, kBarStFull = 13,
+  kBadSmemAlign = 0x7001
+};
+
+struct Barriers {
+  uint64_t* q_full;    // [2]  loader (TMA tx) -> MMA
+  uint64_t* q_empty;   // [2]  epilogue (TMA store has read the staging tile) -> loader
+  uint64_t* kv_full;   // [kKvSlots]
+  uint64_t* kv_empty;  // [kKvSlots]  MMA commit -> loader
+  uint64_t* s_full;    // [2]  MMA commit -> softmax
+  uint64_t* p_full;    // [2]  softmax (4 warps) -> MMA
+  uint64_t* o_full;    // [2]  MMA commit (last P V) -> epilogue
+  uint64_t* o_empty;   // [2]  epilogue (4 warps) -> MMA
+  uint64_t* l_full;    // [2]  softmax (128 threads) -> epilogue
+  uint64_t* l_empty;   // [2]  epilogue (128 threads) -> softmax
+  uint64_t* st_full;   // [2]  epilogue (4 warps: staging tile written) -> the thread issuing the TMA store
+  uint64_t* sched_full;   // [2]  loader -> every consumer role
+  uint64_t* sched_empty;  // [2]  13 consumer arrivals -> loader
+};
+constexpr int kSchedConsumers = 1 + 8 + 4;  // MMA lane, 8 softmax warps, 4 epilogue warps
+
+// Work item of iteration `it` of this CTA for a consumer role (warp-uniform result; < 0 on
+// an expired wait).  `lane_arrives` is true for the one lane per warp that signals consumption.
+__device__ __forceinline__ int consumer_next_work(const FwdParams& p, const Barriers& bars,
+                                                  const volatile int* sched_w, int it, WaitCtx ctx, int role,
+                                                  bool lane_arrives, bool whole_warp) {
+  if (!p.dynamic) return static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
+  if (it == 0) return static_cast<int>(blockIdx.x);
+  const int slot = (it - 1) & 1;
+  bool ok = mbar_wait(&bars.sched_full[slot], ((it - 1) >> 1) & 1, ctx, role | kBarSchedFull);
+  if (whole_warp) ok = __all_sync(0xffffffffu, ok);
+  if (!ok) return -1;
+  const int w = sched_w[slot];
+  if (whole_warp) __syncwarp();
+  if (lane_arrives) mbar_arrive(&bars.sched_empty[slot]);
+  return w;
+}
+
+// ------------------------------------------------------------------------------------------
+// MMA issue helpers (one thread)
+// ------------------------------------------------------------------------------------------
+constexpr uint32_t kIdescQK = make_idesc_bf16(kTile, kTile, 0, 0);     // A = Q, B = K, both K-major
+constexpr uint32_t kIdescPV = make_idesc_bf16(kTile, kHeadDim, 0, 1);  // A = P (tmem), B = V MN-major
+
+// S[128 x 128] = Q[128 x 128] K[128 x 128]^T : 8 steps of 16 along the head dimension.  A half
+// tile holds 64 head-dim elements per row (one 128-byte swizzle row), so a step advances 32 bytes
+// inside the half tile and the second half tile starts 16 KB later.
+__device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint32_t q_smem, uint32_t k_smem) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) {
+    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+    mma_ss(tmem_s, make_smem_desc_sw128(q_smem + off, 16, 1024), make_smem_desc_sw128(k_smem + off, 16, 1024),
+           kIdescQK, kk > 0);
+  }
+}
+// O[128 x 128] (+)= P[128 x 128 keys] V[128 keys x 128] : 8 steps of 16 keys.  P: 8 tensor-memory
+// columns per step (two BF16 per column).  V is MN-major: a key is one 128-byte row of a half
+// tile, 16 keys are 2048 bytes, the second 64 head-dim elements sit 16 KB later (leading offset).
+__device__ __forceinline__ void issue_pv(uint32_t tmem_o, uint32_t tmem_p, uint32_t v_smem, bool accumulate) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) {
+    mma_ts(tmem_o, tmem_p + kk * 8, make_smem_desc_sw128(v_smem + kk * 2048, kHalfBytes, 1024), kIdescPV,
+           (accumulate || kk > 0) ? 1u : 0u);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Roles
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void role_loader(const FwdParams& p, const Barriers& bars, uint8_t* smem,
+                                            volatile int* sched_w, WaitCtx ctx, const CUtensorMap* tm_q,
+                                            const CUtensorMap* tm_k, const CUtensorMap* tm_v) {
+  uint32_t kv_cnt = 0;
+  uint32_t q_cnt[2] = {0, 0};
+  int w = static_cast<int>(blockIdx.x);
+  for (int it = 0; w < p.n_work; ++it) {
+    // fetch the next work item one item ahead and publish it to the other roles
+    int w_next;
+    if (p.dynamic) {
+      const int slot = it & 1;
+      if (!mbar_wait(&bars.sched_empty[slot], ((it >> 1) & 1) ^ 1, ctx, kRoleLoad | kBarSchedEmpty)) return;
+      w_next = static_cast<int>(atomicAdd(p.counter, 1u)) + static_cast<int>(gridDim.x);
+      sched_w[slot] = w_next;
+      mbar_arrive(&bars.sched_full[slot]);
+    } else {
+      w_next = w + static_cast<int>(gridDim.x);
+    }
+    Work wk;
+    decode_work(p, w, wk);
+    int q_pending = 0;  // Q tiles are requested after the first K tile so that K never waits behind them
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      if (wk.n[s] > 0) q_pending |= 1 << s;
+    }
+    for (int j = 0; j < wk.nmax; ++j) {
+      for (int kv = 0; kv < 2; ++kv) {
+        const uint32_t slot = kv_cnt % kKvSlots;
+        const uint32_t par = (kv_cnt / kKvSlots) & 1;
+        if (!mbar_wait(&bars.kv_empty[slot], par ^ 1, ctx, kRoleLoad | kBarKvEmpty)) return;
+        uint8_t* dst = smem + kSmemKv + slot * kTileBytes;
+        mbar_arrive_expect_tx(&bars.kv_full[slot], kTileBytes);
+        const CUtensorMap* tm = kv == 0 ? tm_k : tm_v;
+        tma_load_4d(dst, tm, &bars.kv_full[slot], 0, wk.hkv, j * kTile, wk.b);
+        tma_load_4d(dst + kHalfBytes, tm, &bars.kv_full[slot], 64, wk.hkv, j * kTile, wk.b);
+        ++kv_cnt;
+        if (j == 0 && kv == 0) {
+#pragma unroll
+          for (int s = 0; s < 2; ++s) {
+            if (q_pending & (1 << s)) {
+              if (!mbar_wait(&bars.q_empty[s], (q_cnt[s] & 1) ^ 1, ctx, kRoleLoad | kBarQEmpty)) return;
+              uint8_t* qdst = smem + kSmemQ + s * kTileBytes;
+              mbar_arrive_expect_tx(&bars.q_full[s], kTileBytes);
+              tma_load_4d(qdst, tm_q, &bars.q_full[s], 0, wk.hq[s], wk.row0[s], wk.b);
+              tma_load_4d(qdst + kHalfBytes, tm_q, &bars.q_full[s], 64, wk.hq[s], wk.row0[s], wk.b);
+              ++q_cnt[s];
+            }
+          }
+        }
+      }
+    }
+    w = w_next;
+  }
+}
+
+__device__ __forceinline__ void role_mma(const FwdParams& p, const Barriers& bars, uint8_t* smem,
+                                         const volatile int* sched_w, WaitCtx ctx, uint32_t tmem) {
+  const uint32_t smem_base = smem_u32(smem);
+  uint32_t kv_cnt = 0;
+  uint32_t q_cnt[2] = {0, 0};   // per-stage work items seen (phase of q_full / o_empty)
+  uint32_t sp_cnt[2] = {0, 0};  // per-stage K/V blocks seen (phase of p_full)
+  for (int it = 0;; ++it) {
+    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleMma, true, false);
+    if (w < 0 || w >= p.n_work) return;
+    Work wk;
+    decode_work(p, w, wk);
+    // S_s(0) for both stages
+    {
+      const uint32_t slot = kv_cnt % kKvSlots, par = (kv_cnt / kKvSlots) & 1;
+      if (!mbar_wait(&bars.kv_full[slot], par, ctx, kRoleMma | kBarKvFull)) return;
+      const uint32_t k_smem = smem_base + kSmemKv + slot * kTileBytes;
+#pragma unroll
+      for (int s = 0; s < 2; ++s) {
+        if (wk.n[s] > 0) {
+          if (!mbar_wait(&bars.q_full[s], q_cnt[s] & 1, ctx, kRoleMma | kBarQFull)) return;
+          tc_fence_after_sync();
+          issue_qk(tmem + s * kTile, smem_base + kSmemQ + s * kTileBytes, k_smem);
+          mma_commit(&bars.s_full[s]);
+        }
+      }
+      mma_commit(&bars.kv_empty[slot]);
+      ++kv_cnt;
+    }
+    for (int j = 0; j < wk.nmax; ++j) {
+      const uint32_t vslot = kv_cnt % kKvSlots, vpar = (kv_cnt / kKvSlots) & 1;
+      ++kv_cnt;
+      const bool has_next = (j + 1 < wk.nmax);
+      uint32_t kslot = 0, kpar = 0;
+      if (has_next) {
+        kslot = kv_cnt % kKvSlots;
+        kpar = (kv_cnt / kKvSlots) & 1;
+        ++kv_cnt;
+      }
+      if (!mbar_wait(&bars.kv_full[vslot], vpar, ctx, kRoleMma | kBarKvFull)) return;
+      bool k_ready = false;
+      const uint32_t v_smem = smem_base + kSmemKv + vslot * kTileBytes;
+      const uint32_t k_smem = smem_base + kSmemKv + kslot * kTileBytes;
+#pragma unroll
+      for (int s = 0; s < 2; ++s) {
+        if (j < wk.n[s]) {
+          if (j == 0) {  // the previous item's O_s must have left tensor memory
+            if (!mbar_wait(&bars.o_empty[s], (q_cnt[s] & 1) ^ 1, ctx, kRoleMma | kBarOEmpty)) return;
+          }
+          if (!mbar_wait(&bars.p_full[s], sp_cnt[s] & 1, ctx, kRoleMma | kBarPFull)) return;
+          ++sp_cnt[s];
+          tc_fence_after_sync();
+          issue_pv(tmem + 2 * kTile + s * kTile, tmem + s * kTile, v_smem, j > 0);
+          if (j == wk.n[s] - 1) mma_commit(&bars.o_full[s]);
+          if (j + 1 < wk.n[s]) {
+            if (!k_ready) {
+              if (!mbar_wait(&bars.kv_full[kslot], kpar, ctx, kRoleMma | kBarKvFull)) return;
+              tc_fence_after_sync();
+              k_ready = true;
+            }
+            issue_qk(tmem + s * kTile, smem_base + kSmemQ + s * kTileBytes, k_smem);
+            mma_commit(&bars.s_full[s]);
+          }
+        }
+      }
+      mma_commit(&bars.kv_empty[vslot]);
+      if (has_next) mma_commit(&bars.kv_empty[kslot]);
+    }
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      if (wk.n[s] > 0) ++q_cnt[s];
+    }
+  }
+}
+
+// One softmax thread owns one query row of stage `s`.
+__device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers& bars, uint8_t* smem,
+                                             const volatile int* sched_w, WaitCtx ctx, uint32_t tmem, int s,
+                                             int row_in_tile, int lane) {
+  const uint32_t lane_sel = static_cast<uint32_t>(row_in_tile & ~31) << 16;
+  const uint32_t t_s = tmem + lane_sel + s * kTile;             // S_s, and P_s in its first 64 columns
+  const uint32_t t_o = tmem + lane_sel + 2 * kTile + s * kTile;  // O_s
+  float* stats = reinterpret_cast<float*>(smem + kSmemStats) + s * 2 * kTile;
+  const float c = p.scale_log2;
+  uint32_t s_cnt = 0;  // phase of s_full[s]
+  uint32_t l_cnt = 0;  // phase of l_empty / l_full
+  for (int it = 0;; ++it) {
+    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleSoftmax, lane == 0, true);
+    if (w < 0 || w >= p.n_work) return;
+    Work wk;
+    decode_work(p, w, wk);
+    const int n = wk.n[s];
+    if (n == 0) continue;
+    const int row = wk.row0[s] + row_in_tile;  // global query row (may be >= Sq in a ragged tile)
+    // number of keys this row may see, counted from key 0
+    const int row_limit = p.causal ? min(p.Sk, row + p.off + 1) : p.Sk;
+    // first key index from which a block needs per-element masking for this tile
+    const int tile_clear = p.causal ? min(p.Sk, wk.row0[s] + p.off + 1) : p.Sk;
+    float m_used = -INFINITY;  // row maximum the exponentials are taken against (raw score units)
+    float l = 0.f;             // running sum of exponentials
+    for (int j = 0; j < n; ++j) {
+      bool ok = mbar_wait(&bars.s_full[s], s_cnt & 1, ctx, kRoleSoftmax | kBarSFull);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return;
+      ++s_cnt;
+      tc_fence_after_sync();
+      uint32_t xr[kTile];
+      tmem_ld_x32(t_s + 0, xr + 0);
+      tmem_ld_x32(t_s + 32, xr + 32);
+      tmem_ld_x32(t_s + 64, xr + 64);
+      tmem_ld_x32(t_s + 96, xr + 96);
+      tmem_wait_ld();
+#define X(i) __uint_as_float(xr[(i)])
+      if ((j + 1) * kTile > tile_clear) {  // warp-uniform: some element of this block is masked
+        const int vis = row_limit - j * kTile;  // visible columns of this row in this block
+#pragma unroll
+        for (int i = 0; i < kTile; ++i) {
+          if (i >= vis) xr[i] = 0xff800000u;
+        }
+      }
+      float m0 = X(0), m1 = X(1), m2 = X(2), m3 = X(3);
+#pragma unroll
+      for (int i = 4; i < kTile; i += 8) {
+        m0 = max3(m0, X(i), X(i + 1));
+        m1 = max3(m1, X(i + 2), X(i + 3));
+        if (i + 4 < kTile) {
+          m2 = max3(m2, X(i + 4), X(i + 5));
+          m3 = max3(m3, X(i + 6), X(i + 7));
+        }
+      }
+      const float m_blk = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+      if (j == 0) {
+        m_used = (m_blk == -INFINITY) ? 0.f : m_blk;
+      } else {
+        const float m_new = fmaxf(m_used, m_blk);
+        const bool grow = (m_new - m_used) * c > kRescaleThreshold;
+        if (__any_sync(0xffffffffu, grow)) {
+          // P V of block j-1 has completed (S of block j was issued after it), so O_s is quiescent
+          const float alpha = ex2_approx((m_used - m_new) * c);
+          m_used = m_new;
+          l *= alpha;
+#pragma unroll
+          for (int cc = 0; cc < 8; ++cc) {
+            uint32_t o[16];
+            tmem_ld_x16(t_o + cc * 16, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            tmem_st_x16(t_o + cc * 16, o);
+          }
+        }
+      }
+      const float neg_mc = -m_used * c;
+      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          const float e0 = ex2_approx(fmaf(X(cc * 32 + i + 0), c, neg_mc));
+          const float e1 = ex2_approx(fmaf(X(cc * 32 + i + 1), c, neg_mc));
+          const float e2 = ex2_approx(fmaf(X(cc * 32 + i + 2), c, neg_mc));
+          const float e3 = ex2_approx(fmaf(X(cc * 32 + i + 3), c, neg_mc));
+          l0 += e0;
+          l1 += e1;
+          l2 += e2;
+          l3 += e3;
+          pk[i / 2] = pack_bf16x2(e0, e1);
+          pk[i / 2 + 1] = pack_bf16x2(e2, e3);
+        }
+        tmem_st_x16(t_s + cc * 16, pk);
+      }
+#undef X
+      l += (l0 + l1) + (l2 + l3);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      if (lane == 0) mbar_arrive(&bars.p_full[s]);
+    }
+    // hand the row statistics to the epilogue warps
+    bool ok = mbar_wait(&bars.l_empty[s], (l_cnt & 1) ^ 1, ctx, kRoleSoftmax | kBarLEmpty);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) return;
+    stats[row_in_tile] = l;
+    stats[kTile + row_in_tile] = m_used;
+    mbar_arrive(&bars.l_full[s]);
+    ++l_cnt;
+  }
+}
+
+__device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers& bars, uint8_t* smem,
+                                              const volatile int* sched_w, WaitCtx ctx, uint32_t tmem,
+                                              int row_in_tile, int lane, const CUtensorMap* tm_o) {
+  const uint32_t lane_sel = static_cast<uint32_t>(row_in_tile & ~31) << 16;
+  uint32_t cnt[2] = {0, 0};
+  for (int it = 0;; ++it) {
+    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleEpilogue, lane == 0, true);
+    if (w < 0 || w >= p.n_work) return;
+    Work wk;
+    decode_work(p, w, wk);
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      if (wk.n[s] == 0) continue;
+      const float* stats = reinterpret_cast<const float*>(smem + kSmemStats) + s * 2 * kTile;
+      bool ok = mbar_wait(&bars.l_full[s], cnt[s] & 1, ctx, kRoleEpilogue | kBarLFull);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return;
+      const float l = stats[row_in_tile];
+      const float m_used = stats[kTile + row_in_tile];
+      mbar_arrive(&bars.l_empty[s]);
+      ok = mbar_wait(&bars.o_full[s], cnt[s] & 1, ctx, kRoleEpilogue | kBarOFull);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return;
+      ++cnt[s];
+      tc_fence_after_sync();
+      const float inv_l = 1.0f / l;
+      uint8_t* stage = smem + kSmemQ + s * kTileBytes;  // the Q_s tile is dead once o_full[s] fired
+      const uint32_t t_o = tmem + lane_sel + 2 * kTile + s * kTile;
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t o[32];
+        tmem_ld_x32(t_o + cc * 32, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint4 val;
+          val.x = pack_bf16x2(__uint_as_float(o[ch * 8 + 0]) * inv_l, __uint_as_float(o[ch * 8 + 1]) * inv_l);
+          val.y = pack_bf16x2(__uint_as_float(o[ch * 8 + 2]) * inv_l, __uint_as_float(o[ch * 8 + 3]) * inv_l);
+          val.z = pack_bf16x2(__uint_as_float(o[ch * 8 + 4]) * inv_l, __uint_as_float(o[ch * 8 + 5]) * inv_l);
+          val.w = pack_bf16x2(__uint_as_float(o[ch * 8 + 6]) * inv_l, __uint_as_float(o[ch * 8 + 7]) * inv_l);
+          const int chunk = cc * 4 + ch;  // 16-byte chunk of the 256-byte row
+          uint8_t* dst = stage + (chunk >> 3) * kHalfBytes + row_in_tile * 128 +
+                         (((chunk & 7) ^ (row_in_tile & 7)) << 4);
+          *reinterpret_cast<uint4*>(dst) = val;
+        }
+      }
+      tc_fence_before_sync();
+      if (lane == 0) mbar_arrive(&bars.o_empty[s]);
+      const int row = wk.row0[s] + row_in_tile;
+      if (p.lse != nullptr && row < p.Sq) {
+        p.lse[(static_cast<size_t>(wk.b) * p.Hq + wk.hq[s]) * p.Sq + row] = m_used * p.scale + logf(l);
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars.st_full[s]);
+      if (row_in_tile == s * 32) {
+        // cnt[s] was advanced above: this item's phase of st_full[s] is (cnt[s] - 1) & 1
+        if (mbar_wait(&bars.st_full[s], (cnt[s] & 1) ^ 1, ctx, kRoleEpilogue | kBarStFull)) {
+          tma_store_4d(tm_o, stage, 0, wk.hq[s], wk.row0[s], wk.b);
+          tma_store_4d(tm_o, stage + kHalfBytes, 64, wk.hq[s], wk.row0[s], wk.b);
+          tma_store_commit();
+          tma_store_wait_read0();
+          mbar_arrive(&bars.q_empty[s]);
+        }
+      }
+    }
+  }
+  // global writes of the bulk stores complete before the kernel ends
+}
+
+// ------------------------------------------------------------------------------------------
+// Kernel
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                const FwdParams p) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint64_t* bar_mem = reinterpret_cast<uint64_t*>(smem + kSmemBars);
+  Barriers bars;
+  bars.q_full = bar_mem;
+  bars.q_empty = bars.q_full + 2;
+  bars.kv_full = bars.q_empty + 2;
+  bars.kv_empty = bars.kv_full + kKvSlots;
+  bars.s_full = bars.kv_empty + kKvSlots;
+  bars.p_full = bars.s_full + 2;
+  bars.o_full = bars.p_full + 2;
+  bars.o_empty = bars.o_full + 2;
+  bars.l_full = bars.o_empty + 2;
+  bars.l_empty = bars.l_full + 2;
+  bars.st_full = bars.l_empty + 2;
+  bars.sched_full = bars.st_full + 2;
+  bars.sched_empty = bars.sched_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kSmemMisc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kSmemMisc + 4);
+  volatile int* sched_w = reinterpret_cast<volatile int*>(smem + kSmemMisc + 8);
+  const WaitCtx ctx{abort_flag, p.status};
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const int lane = tid & 31;
+
+  if ((smem_u32(smem) & 1023u) != 0) {  // the swizzled tiles need a 1024-byte aligned base
+    if (tid == 0 && atomicCAS(p.status, 0, kBadSmemAlign) == 0) p.status[1] = static_cast<int>(blockIdx.x);
+    return;
+  }
+  if (tid == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars.q_full[i], 1);
+      mbar_init(&bars.q_empty[i], 1);
+      mbar_init(&bars.s_full[i], 1);
+      mbar_init(&bars.p_full[i], 4);
+      mbar_init(&bars.o_full[i], 1);
+      mbar_init(&bars.o_empty[i], 4);
+      mbar_init(&bars.l_full[i], kTile);
+      mbar_init(&bars.l_empty[i], kTile);
+      mbar_init(&bars.st_full[i], 4);
+      mbar_init(&bars.sched_full[i], 1);
+      mbar_init(&bars.sched_empty[i], kSchedConsumers);
+    }
+    for (int i = 0; i < kKvSlots; ++i) {
+      mbar_init(&bars.kv_full[i], 1);
+      mbar_init(&bars.kv_empty[i], 1);
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 12) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  if (warp == 13 && lane == 0) {
+    tma_prefetch_desc(&tm_q);
+    tma_prefetch_desc(&tm_k);
+    tma_prefetch_desc(&tm_v);
+    tma_prefetch_desc(&tm_o);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp < 8) {
+    reg_alloc<ATTN_REGS_SOFTMAX>();
+    role_softmax(p, bars, smem, sched_w, ctx, tmem, warp >> 2, tid & 127, lane);
+  } else if (warp < 12) {
+    reg_dealloc<ATTN_REGS_EPILOGUE>();
+    role_epilogue(p, bars, smem, sched_w, ctx, tmem, tid & 127, lane, &tm_o);
+    tma_store_wait_all0();
+  } else {
+    reg_dealloc<ATTN_REGS_OTHER>();
+    if (warp == 12) {
+      if (lane == 0) role_mma(p, bars, smem, sched_w, ctx, tmem);
+    } else if (warp == 13) {
+      if (lane == 0) {
+        role_loader(p, bars, smem, sched_w, ctx, &tm_q, &tm_k, &tm_v);
+        if (*abort_flag) {  // let loads in flight land before the CTA's shared memory is released
+          const uint64_t t0 = global_timer_ns();
+          while (global_timer_ns() - t0 < 1000000ull) {
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 12) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace attn
