@@ -28,7 +28,7 @@ typedef enum {
   ATTN_OK = 0,
   ATTN_ERR_NULL = 1,        /* a required pointer is NULL */
   ATTN_ERR_SHAPE = 2,       /* a dimension is <= 0, or Hq is not a multiple of Hkv */
-  ATTN_ERR_UNSUPPORTED = 3, /* D != 128; causal with Sq > Sk; scale not finite or < 0 */
+  ATTN_ERR_UNSUPPORTED = 3, /* D != 128; causal with Sq > Sk; scale not finite or <= 0 */
   ATTN_ERR_ALIGN = 4,       /* q, k, v or o not 16-byte aligned; lse not 4-byte aligned */
   ATTN_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed (descriptor, launch, copy) */
   ATTN_ERR_ARCH = 6,        /* the current device is not compute capability 10.x */
@@ -54,7 +54,7 @@ typedef enum {
  *   D        must be 128
  *   causal   0: every key is visible.  non-zero: key j is visible to query i iff
  *            j <= i + (Sk - Sq)  (lower-triangular when Sq == Sk); requires Sq <= Sk
- *   scale    multiplies Q K^T; finite and >= 0 (callers normally pass 1/sqrt(D))
+ *   scale    multiplies Q K^T; finite and > 0 (callers normally pass 1/sqrt(D))
  *   stream   cudaStream_t (NULL = default stream)
  *
  * o must not alias q, k or v.  Distinct streams may call concurrently.  The first
@@ -91,6 +91,27 @@ attn_status_t attn_release_host_staging(void);
  *   "max_ctas"    0 = one per SM (default), else an upper bound on persistent CTAs
  */
 attn_status_t attn_set_option(const char* name, int value);
+
+/*
+ * attn_plan / attn_plan_item -- host-only introspection of the tile scheduler (Section 2.2's
+ * "processes key blocks sequentially" per query tile, and the causal case where some key
+ * blocks are fully masked and skipped).  No device is touched.
+ *
+ * attn_plan fills plan[0..5] = { n_work, pair_heads, items_per_group, n_q_tiles,
+ * n_kv_blocks, ctas } for a problem, where `ctas` is the grid a launch on a device with
+ * `sm_count` SMs would use under the current options.  A work item is two 128-row query
+ * tiles ("stages") that share one stream of K/V tiles: two consecutive row tiles of one
+ * query head (pair_heads = 0), or the same row tile of two query heads that share a KV
+ * head (pair_heads = 1, used when Hq / Hkv is even).
+ *
+ * attn_plan_item fills item[0..7] = { b, hkv, hq0, hq1, row0_0, row0_1, n_blocks_0,
+ * n_blocks_1 } for work item `w` in launch order (causal: longest items first inside each
+ * head).  n_blocks_s = 0 marks an unused stage (its rows lie beyond Sq).
+ * Both return ATTN_ERR_SHAPE / ATTN_ERR_UNSUPPORTED like attn_fwd, ATTN_ERR_SHAPE for w
+ * out of range.
+ */
+attn_status_t attn_plan(int B, int Hq, int Hkv, int Sq, int Sk, int D, int causal, int sm_count, int* plan);
+attn_status_t attn_plan_item(int B, int Hq, int Hkv, int Sq, int Sk, int D, int causal, int w, int* item);
 
 /* Human-readable name of a status code (static storage). */
 const char* attn_status_str(attn_status_t status);

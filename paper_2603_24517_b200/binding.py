@@ -21,7 +21,8 @@ STATUS_NAMES = {
     5: "ATTN_ERR_CUDA", 6: "ATTN_ERR_ARCH", 7: "ATTN_ERR_TIMEOUT",
 }
 EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_host", "attn_release_host_staging", "attn_set_option",
-                    "attn_status_str", "attn_version", "attn_last_device_status")
+                    "attn_plan", "attn_plan_item", "attn_status_str", "attn_version",
+                    "attn_last_device_status")
 
 _lib = None
 
@@ -51,6 +52,10 @@ def load_library() -> ctypes.CDLL:
     lib.attn_release_host_staging.restype = ci
     lib.attn_set_option.argtypes = [ctypes.c_char_p, ci]
     lib.attn_set_option.restype = ci
+    lib.attn_plan.argtypes = [ci] * 8 + [ctypes.POINTER(ci)]
+    lib.attn_plan.restype = ci
+    lib.attn_plan_item.argtypes = [ci] * 8 + [ctypes.POINTER(ci)]
+    lib.attn_plan_item.restype = ci
     lib.attn_status_str.argtypes = [ci]
     lib.attn_status_str.restype = ctypes.c_char_p
     lib.attn_version.argtypes = []
@@ -119,6 +124,26 @@ def attn_set_option(name: str, value: int) -> None:
     st = load_library().attn_set_option(name.encode(), int(value))
     if st != ATTN_OK:
         raise AttnError(st, f"attn_set_option({name}={value})")
+
+
+def attn_plan(B, Hq, Hkv, Sq, Sk, D, causal, sm_count) -> dict:
+    """Host-only: the tile scheduler's decomposition of a problem (see include/attn.h)."""
+    out = (ctypes.c_int * 6)()
+    st = load_library().attn_plan(B, Hq, Hkv, Sq, Sk, D, int(bool(causal)), sm_count, out)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_plan")
+    keys = ("n_work", "pair_heads", "items_per_group", "n_q_tiles", "n_kv_blocks", "ctas")
+    return dict(zip(keys, list(out)))
+
+
+def attn_plan_item(B, Hq, Hkv, Sq, Sk, D, causal, w) -> dict:
+    """Host-only: work item ``w`` in launch order (see include/attn.h)."""
+    out = (ctypes.c_int * 8)()
+    st = load_library().attn_plan_item(B, Hq, Hkv, Sq, Sk, D, int(bool(causal)), w, out)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_plan_item")
+    keys = ("b", "hkv", "hq0", "hq1", "row0_0", "row0_1", "n_blocks_0", "n_blocks_1")
+    return dict(zip(keys, list(out)))
 
 
 def attn_status_str(status: int) -> str:

@@ -120,9 +120,72 @@ attn_status_t check_args(const void* q, const void* k, const void* v, void* o, c
   return ATTN_OK;
 }
 
+// Problem geometry and work decomposition (no device access).
+void fill_plan(FwdParams* p, int B, int Hq, int Hkv, int Sq, int Sk, int causal) {
+  std::memset(p, 0, sizeof(*p));
+  p->B = B; p->Hq = Hq; p->Hkv = Hkv; p->Sq = Sq; p->Sk = Sk;
+  p->group = Hq / Hkv;
+  p->causal = causal ? 1 : 0;
+  p->off = Sk - Sq;
+  p->n_qt = (Sq + attn::kTile - 1) / attn::kTile;
+  p->n_kb = (Sk + attn::kTile - 1) / attn::kTile;
+  p->pair_heads = (p->group % 2 == 0) ? 1 : 0;
+  if (p->pair_heads) {
+    p->items_per_group = p->n_qt * (p->group / 2);
+    p->n_work = B * Hkv * p->items_per_group;
+  } else {
+    p->items_per_group = (p->n_qt + 1) / 2;
+    p->n_work = B * Hq * p->items_per_group;
+  }
+  p->dynamic = (g_opt_scheduler.load() == 2) ? 1 : 0;
+}
+
+int plan_grid(const FwdParams& p, int sm_count) {
+  int grid = p.n_work;
+  if (g_opt_scheduler.load() != 0) {
+    int cap = sm_count;
+    const int max_ctas = g_opt_max_ctas.load();
+    if (max_ctas > 0 && max_ctas < cap) cap = max_ctas;
+    if (grid > cap) grid = cap;
+  }
+  return grid;
+}
+
 }  // namespace
 
 extern "C" {
+
+attn_status_t attn_plan(int B, int Hq, int Hkv, int Sq, int Sk, int D, int causal, int sm_count, int* plan) {
+  if (plan == nullptr) return ATTN_ERR_NULL;
+  int dummy = 0;
+  attn_status_t st = check_args(&dummy, &dummy, &dummy, &dummy, nullptr, B, Hq, Hkv, Sq, Sk, D, causal, 1.0f, false);
+  if (st != ATTN_OK) return st;
+  if (sm_count <= 0) return ATTN_ERR_SHAPE;
+  FwdParams p;
+  fill_plan(&p, B, Hq, Hkv, Sq, Sk, causal);
+  plan[0] = p.n_work;
+  plan[1] = p.pair_heads;
+  plan[2] = p.items_per_group;
+  plan[3] = p.n_qt;
+  plan[4] = p.n_kb;
+  plan[5] = plan_grid(p, sm_count);
+  return ATTN_OK;
+}
+
+attn_status_t attn_plan_item(int B, int Hq, int Hkv, int Sq, int Sk, int D, int causal, int w, int* item) {
+  if (item == nullptr) return ATTN_ERR_NULL;
+  int dummy = 0;
+  attn_status_t st = check_args(&dummy, &dummy, &dummy, &dummy, nullptr, B, Hq, Hkv, Sq, Sk, D, causal, 1.0f, false);
+  if (st != ATTN_OK) return st;
+  FwdParams p;
+  fill_plan(&p, B, Hq, Hkv, Sq, Sk, causal);
+  if (w < 0 || w >= p.n_work) return ATTN_ERR_SHAPE;
+  attn::Work wk;
+  attn::decode_work(p, w, wk);
+  item[0] = wk.b; item[1] = wk.hkv; item[2] = wk.hq[0]; item[3] = wk.hq[1];
+  item[4] = wk.row0[0]; item[5] = wk.row0[1]; item[6] = wk.n[0]; item[7] = wk.n[1];
+  return ATTN_OK;
+}
 
 attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
                        int Sq, int Sk, int D, int causal, float scale, void* stream) {
@@ -137,35 +200,12 @@ attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, flo
     return ATTN_ERR_CUDA;
 
   FwdParams p;
-  std::memset(&p, 0, sizeof(p));
-  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
-  p.group = Hq / Hkv;
-  p.causal = causal ? 1 : 0;
-  p.off = Sk - Sq;
-  p.n_qt = (Sq + attn::kTile - 1) / attn::kTile;
-  p.n_kb = (Sk + attn::kTile - 1) / attn::kTile;
-  p.pair_heads = (p.group % 2 == 0) ? 1 : 0;
-  if (p.pair_heads) {
-    p.items_per_group = p.n_qt * (p.group / 2);
-    p.n_work = B * Hkv * p.items_per_group;
-  } else {
-    p.items_per_group = (p.n_qt + 1) / 2;
-    p.n_work = B * Hq * p.items_per_group;
-  }
+  fill_plan(&p, B, Hq, Hkv, Sq, Sk, causal);
   p.scale = scale;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.lse = lse;
   p.status = dev->status;
-
-  const int sched = g_opt_scheduler.load();
-  int grid = p.n_work;
-  if (sched != 0) {
-    int cap = dev->sm_count;
-    const int max_ctas = g_opt_max_ctas.load();
-    if (max_ctas > 0 && max_ctas < cap) cap = max_ctas;
-    if (grid > cap) grid = cap;
-  }
-  p.dynamic = (sched == 2) ? 1 : 0;
+  const int grid = plan_grid(p, dev->sm_count);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (p.dynamic) {
     const unsigned int slot = dev->next_slot.fetch_add(1) % kCounterSlots;

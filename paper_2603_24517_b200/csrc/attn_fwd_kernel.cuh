@@ -77,7 +77,7 @@ struct Work {
   int nmax;
 };
 
-__device__ __forceinline__ void decode_work(const FwdParams& p, int w, Work& wk) {
+__host__ __device__ __forceinline__ void decode_work(const FwdParams& p, int w, Work& wk) {
   const int grp = w / p.items_per_group;
   const int r = w - grp * p.items_per_group;
   if (p.pair_heads) {
@@ -103,13 +103,14 @@ __device__ __forceinline__ void decode_work(const FwdParams& p, int w, Work& wk)
     if (wk.row0[s] >= p.Sq) {
       wk.n[s] = 0;
     } else if (p.causal) {
-      const int last_row = min(wk.row0[s] + kTile, p.Sq) - 1;
-      wk.n[s] = min(p.n_kb, (last_row + p.off) / kTile + 1);
+      const int row_end = wk.row0[s] + kTile < p.Sq ? wk.row0[s] + kTile : p.Sq;
+      const int need = (row_end - 1 + p.off) / kTile + 1;
+      wk.n[s] = need < p.n_kb ? need : p.n_kb;
     } else {
       wk.n[s] = p.n_kb;
     }
   }
-  wk.nmax = max(wk.n[0], wk.n[1]);
+  wk.nmax = wk.n[0] > wk.n[1] ? wk.n[0] : wk.n[1];
 }
 
 // ------------------------------------------------------------------------------------------

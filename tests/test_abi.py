@@ -1,0 +1,84 @@
+"""The C-ABI shared library loads without a GPU, exports every symbol that include/attn.h
+declares, and rejects bad arguments before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2603_24517_b200 as lib
+from paper_2603_24517_b200 import binding
+from paper_2603_24517_b200 import build as lib_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def cdll():
+    lib_build.build()
+    return lib.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "attn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(attn_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(cdll):
+    names = declared_functions()
+    assert "attn_fwd" in names and "attn_fwd_host" in names and len(names) >= 9
+    for name in names:
+        assert hasattr(cdll, name), f"{name} declared in include/attn.h but not exported"
+    assert set(names) == set(binding.EXPORTED_SYMBOLS)
+
+
+def test_version_and_status_strings(cdll):
+    assert lib.attn_version() >= 100
+    for code, name in binding.STATUS_NAMES.items():
+        assert lib.attn_status_str(code) == name
+    assert lib.attn_status_str(99) == "ATTN_ERR_UNKNOWN"
+
+
+def _fwd(cdll, q=16, k=16, v=16, o=16, lse=0, B=1, Hq=2, Hkv=2, Sq=128, Sk=128, D=128, causal=0, scale=0.1):
+    return cdll.attn_fwd(q, k, v, o, lse or None, B, Hq, Hkv, Sq, Sk, D, causal, scale, None)
+
+
+def test_argument_errors_need_no_device(cdll):
+    assert _fwd(cdll, q=0) == 1            # ATTN_ERR_NULL
+    assert _fwd(cdll, o=0) == 1
+    assert _fwd(cdll, B=0) == 2            # ATTN_ERR_SHAPE
+    assert _fwd(cdll, Sk=-5) == 2
+    assert _fwd(cdll, Hq=3, Hkv=2) == 2
+    assert _fwd(cdll, D=64) == 3           # ATTN_ERR_UNSUPPORTED
+    assert _fwd(cdll, causal=1, Sq=256, Sk=128) == 3
+    assert _fwd(cdll, scale=float("nan")) == 3
+    assert _fwd(cdll, scale=float("inf")) == 3
+    assert _fwd(cdll, scale=-1.0) == 3
+    assert _fwd(cdll, scale=0.0) == 3
+    assert _fwd(cdll, q=24) == 4           # ATTN_ERR_ALIGN
+    assert _fwd(cdll, lse=18) == 4
+    # host entry point: same shape checks, no alignment requirement
+    assert cdll.attn_fwd_host(None, 16, 16, 16, None, 1, 2, 2, 128, 128, 128, 0, 0.1, None) == 1
+    assert cdll.attn_fwd_host(16, 16, 16, 16, None, 1, 2, 2, 128, 128, 96, 0, 0.1, None) == 3
+
+
+def test_options(cdll):
+    assert cdll.attn_set_option(b"scheduler", 3) == 3
+    assert cdll.attn_set_option(b"no_such_option", 1) == 3
+    assert cdll.attn_set_option(None, 1) == 1
+    for v in (0, 1, 2):
+        assert cdll.attn_set_option(b"scheduler", v) == 0
+    assert cdll.attn_set_option(b"max_ctas", -1) == 3
+    assert cdll.attn_set_option(b"max_ctas", 0) == 0
+
+
+def test_last_device_status_null(cdll):
+    assert cdll.attn_last_device_status(None, None) == 1
+
+
+def test_missing_library_is_loud(monkeypatch):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libattn_b200.so"))
+    with pytest.raises(ImportError):
+        binding.load_library()

@@ -1,0 +1,220 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU fp64 oracle, element by
+element on the same seeded BF16 inputs.
+
+Tolerances (max-norm, absolute): |dO| <= 2e-2 and |dLSE| <= 1e-3.  O is rounded to BF16
+(half an ulp is 1.6e-2 for |O| in [4, 8)), P is rounded to BF16 before P V, and the
+exponentials come from ex2.approx; LSE is fp32 end to end.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2603_24517_b200 as lib
+from paper_2603_24517_b200 import build as lib_build
+from oracle import attn_oracle as orc
+from workloads import all_workloads, bf16_bits, bits_to_float64, make_qkv, make_workload_inputs, sample_rows
+
+pytestmark = pytest.mark.gpu
+
+TOL_O = 2e-2
+TOL_LSE = 1e-3
+SCALE = float(np.float32(1.0 / math.sqrt(128)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _library():
+    lib_build.build()
+    lib.load_library()
+    lib.attn_set_option("scheduler", 2)
+    lib.attn_set_option("max_ctas", 0)
+    yield
+    lib.attn_set_option("scheduler", 2)
+    lib.attn_set_option("max_ctas", 0)
+
+
+def run_gpu(q, k, v, causal, scale, want_lse=True, stream=None):
+    """q, k, v: CPU bf16 tensors.  Outputs are poison-filled so an unwritten element shows."""
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    o = torch.full_like(qd, float("nan"))
+    B, Sq, Hq, _ = q.shape
+    lse = torch.full((B, Hq, Sq), float("nan"), device="cuda", dtype=torch.float32) if want_lse else None
+    if stream is None:
+        lib.attn_fwd(qd, kd, vd, o, lse, causal, scale)
+    else:
+        with torch.cuda.stream(stream):
+            lib.attn_fwd(qd, kd, vd, o, lse, causal, scale)
+        stream.synchronize()
+    torch.cuda.synchronize()
+    st, code, detail = lib.attn_last_device_status()
+    assert (st, code) == (0, 0), f"device status {st} code {code:#x} detail {detail}"
+    return o.cpu(), (None if lse is None else lse.cpu())
+
+
+def check_full(q, k, v, causal, scale, o, lse):
+    o_ref, lse_ref = orc.attention_full(bf16_bits(q), bf16_bits(k), bf16_bits(v), causal, scale)
+    o64 = bits_to_float64(bf16_bits(o))
+    assert not np.isnan(o64).any()
+    d_o = np.abs(o64 - o_ref).max()
+    assert d_o <= TOL_O, f"max|dO| = {d_o}"
+    if lse is not None:
+        l64 = lse.numpy().astype(np.float64)
+        assert not np.isnan(l64).any()
+        d_l = np.abs(l64 - lse_ref).max()
+        assert d_l <= TOL_LSE, f"max|dLSE| = {d_l}"
+
+
+def check_rows(q, k, v, causal, scale, o, lse, rows):
+    o_ref, lse_ref = orc.attention_rows(bf16_bits(q), bf16_bits(k), bf16_bits(v), causal, scale, rows)
+    o64 = bits_to_float64(bf16_bits(o))[rows[:, 0], rows[:, 2], rows[:, 1]]
+    l64 = lse.numpy().astype(np.float64)[rows[:, 0], rows[:, 1], rows[:, 2]]
+    assert not np.isnan(o64).any() and not np.isnan(l64).any()
+    d_o, d_l = np.abs(o64 - o_ref).max(), np.abs(l64 - lse_ref).max()
+    assert d_o <= TOL_O, f"max|dO| = {d_o}"
+    assert d_l <= TOL_LSE, f"max|dLSE| = {d_l}"
+
+
+# B, Hq, Hkv, Sq, Sk, causal -- sizes the oracle finishes in seconds, spanning several tiles,
+# ragged tails, Sq != Sk, odd and even GQA groups, and the degenerate one-key / one-row cases.
+SMALL = [
+    (1, 2, 2, 512, 512, False),       # the small configuration of the benchmark list
+    (1, 2, 2, 512, 512, True),
+    (1, 1, 1, 128, 128, True),        # one tile: the diagonal block is also the first block
+    (1, 1, 1, 256, 256, True),
+    (1, 1, 1, 1, 1, False),
+    (1, 1, 1, 1, 1, True),
+    (1, 2, 2, 1, 700, True),          # one query row at the end of a long key sequence
+    (1, 2, 2, 300, 1, False),         # a single key: O = V row
+    (2, 3, 3, 384, 640, False),
+    (2, 3, 3, 384, 640, True),        # Sq < Sk, bottom-right aligned mask
+    (1, 2, 2, 100, 100, True),        # shorter than a tile
+    (1, 2, 1, 77, 333, True),
+    (1, 3, 1, 300, 300, True),        # odd GQA group: stages pair row tiles
+    (1, 6, 2, 257, 511, True),
+    (2, 2, 2, 129, 257, False),       # one row past a tile edge
+    (1, 8, 2, 256, 512, False),       # group 4: stages pair query heads
+    (1, 8, 1, 384, 384, True),        # group 8
+    (5, 2, 2, 200, 136, False),
+    (1, 4, 4, 1280, 1280, True),      # more K/V blocks than ring slots, several items per CTA
+]
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,causal", SMALL)
+def test_small_cases_match_oracle_everywhere(B, Hq, Hkv, Sq, Sk, causal):
+    q, k, v = make_qkv(B, Hq, Hkv, Sq, Sk, 128, seed=7000 + Sq + Sk)
+    o, lse = run_gpu(q, k, v, causal, SCALE)
+    check_full(q, k, v, causal, SCALE, o, lse)
+
+
+@pytest.mark.parametrize("sched", [0, 1, 2])
+@pytest.mark.parametrize("max_ctas", [0, 3])
+def test_every_scheduler_mode(sched, max_ctas):
+    lib.attn_set_option("scheduler", sched)
+    lib.attn_set_option("max_ctas", max_ctas)
+    try:
+        for (B, Hq, Hkv, Sq, Sk, causal) in [(2, 4, 4, 640, 640, True), (1, 8, 2, 500, 900, False)]:
+            q, k, v = make_qkv(B, Hq, Hkv, Sq, Sk, 128, seed=7100)
+            o, lse = run_gpu(q, k, v, causal, SCALE)
+            check_full(q, k, v, causal, SCALE, o, lse)
+    finally:
+        lib.attn_set_option("scheduler", 2)
+        lib.attn_set_option("max_ctas", 0)
+
+
+@pytest.mark.parametrize("scale,gain", [(0.5, 1.0), (1e-3, 1.0), (SCALE, 4.0), (SCALE, 8.0)])
+def test_scales_and_peaked_rows(scale, gain):
+    """Large score magnitudes move the row maximum by more than the rescale threshold, so the
+    accumulator-rescale path runs; tiny scales make softmax nearly uniform."""
+    q, k, v = make_qkv(1, 2, 2, 1024, 1024, 128, seed=7200, q_gain=gain)
+    scale = float(np.float32(scale))
+    for causal in (False, True):
+        o, lse = run_gpu(q, k, v, causal, scale)
+        check_full(q, k, v, causal, scale, o, lse)
+
+
+def test_increasing_scores_force_rescales():
+    """Keys ordered so that every block raises every row's maximum by far more than the
+    threshold: each K/V block triggers a rescale of O."""
+    B, H, S = 1, 1, 1024
+    q = torch.ones((B, S, H, 128), dtype=torch.bfloat16)
+    ramp = (torch.arange(S, dtype=torch.float32) / 8.0).reshape(1, S, 1, 1)
+    k = (ramp * torch.ones((1, 1, 1, 128))).to(torch.bfloat16)
+    _, _, v = make_qkv(B, H, H, S, S, 128, seed=7300)
+    scale = float(np.float32(1.0 / 16))
+    for causal in (False, True):
+        o, lse = run_gpu(q, k, v, causal, scale)
+        check_full(q, k, v, causal, scale, o, lse)
+
+
+def test_lse_may_be_null_and_stream_is_honoured():
+    q, k, v = make_qkv(1, 2, 2, 384, 384, 128, seed=7400)
+    o1, _ = run_gpu(q, k, v, True, SCALE, want_lse=False)
+    o2, lse2 = run_gpu(q, k, v, True, SCALE, stream=torch.cuda.Stream())
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+    check_full(q, k, v, True, SCALE, o2, lse2)
+
+
+def test_bitwise_deterministic():
+    q, k, v = make_qkv(2, 4, 2, 1000, 1000, 128, seed=7500)
+    outs = [run_gpu(q, k, v, True, SCALE) for _ in range(3)]
+    for o, lse in outs[1:]:
+        assert torch.equal(o.view(torch.int16), outs[0][0].view(torch.int16))
+        assert torch.equal(lse.view(torch.int32), outs[0][1].view(torch.int32))
+
+
+def test_zero_q_gives_prefix_means_at_scale():
+    """Q = 0: O is the mean of the visible V rows and LSE = log(#visible keys), a closed form
+    that checks masking and block counts of every row at a size the oracle cannot sweep."""
+    B, H, S = 1, 4, 8192
+    _, k, v = make_qkv(B, H, H, S, S, 128, seed=7600)
+    q = torch.zeros((B, S, H, 128), dtype=torch.bfloat16)
+    o, lse = run_gpu(q, k, v, True, SCALE)
+    v64 = bits_to_float64(bf16_bits(v))
+    n = np.arange(1, S + 1, dtype=np.float64).reshape(1, S, 1, 1)
+    ref = np.cumsum(v64, axis=1) / n
+    assert np.abs(bits_to_float64(bf16_bits(o)) - ref).max() <= TOL_O
+    ref_lse = np.log(np.arange(1, S + 1, dtype=np.float64)).reshape(1, 1, S)
+    assert np.abs(lse.numpy().astype(np.float64) - ref_lse).max() <= TOL_LSE
+
+
+def test_host_entry_point_matches_device_entry_point():
+    q, k, v = make_qkv(2, 4, 2, 300, 520, 128, seed=7700)
+    o_dev, lse_dev = run_gpu(q, k, v, True, SCALE)
+    qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+    o = torch.empty_like(q).pin_memory()
+    lse = torch.empty((2, 4, 300), dtype=torch.float32).pin_memory()
+    lib.attn_fwd_host(qh, kh, vh, o, lse, True, SCALE)
+    assert torch.equal(o.view(torch.int16), o_dev.view(torch.int16))
+    assert torch.equal(lse, lse_dev)
+    lib.attn_release_host_staging()
+
+
+def test_error_statuses_on_device_tensors():
+    q, k, v = (t.cuda() for t in make_qkv(1, 2, 2, 256, 128, 128, seed=7800))
+    o = torch.empty_like(q)
+    assert lib.attn_fwd_status(q, k, v, o, None, True, SCALE) == 3     # causal with Sq > Sk
+    assert lib.attn_fwd_status(q, k, v, o, None, False, -1.0) == 3
+    assert lib.attn_fwd_status(q, k, v, o, None, False, SCALE) == 0
+    torch.cuda.synchronize()
+
+
+# ---- the benchmark workloads at full size, in the launch configuration bench.py times --------
+FULL = [n for n in all_workloads() if n != "tiny_mha"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_benchmark_workloads_on_sampled_rows(name):
+    w = all_workloads()[name]
+    q, k, v = make_workload_inputs(w)
+    o, lse = run_gpu(q, k, v, w.causal, w.scale)
+    n_rows = 768 if w.Sk >= 32768 else 1536
+    rows = sample_rows(w.B, w.Hq, w.Sq, n_rows, seed=w.seed)
+    check_rows(q, k, v, w.causal, w.scale, o, lse, rows)
+
+
+def test_tiny_workload_in_full():
+    w = all_workloads()["tiny_mha"]
+    q, k, v = make_workload_inputs(w)
+    o, lse = run_gpu(q, k, v, w.causal, w.scale)
+    check_full(q, k, v, w.causal, w.scale, o, lse)

@@ -1,0 +1,96 @@
+"""Host logic of the tile scheduler, checked against brute force on the CPU: every 128-row
+query tile of every (batch, query head) is covered exactly once, GQA stages share a KV head,
+and a stage visits exactly the K/V blocks that hold at least one visible key (paper,
+Section 2.2: fully masked key blocks are skipped under the causal mask)."""
+import math
+
+import pytest
+
+import paper_2603_24517_b200 as lib
+from paper_2603_24517_b200 import build as lib_build
+
+TILE = 128
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    lib_build.build()
+    lib.attn_set_option("scheduler", 2)
+    lib.attn_set_option("max_ctas", 0)
+
+
+def visible_blocks_brute(row0, Sq, Sk, causal):
+    rows = range(row0, min(row0 + TILE, Sq))
+    if not causal:
+        return math.ceil(Sk / TILE)
+    last_key = max(min(Sk - 1, i + Sk - Sq) for i in rows)
+    return last_key // TILE + 1
+
+
+CASES = [
+    (1, 2, 2, 512, 512, False), (1, 2, 2, 512, 512, True), (2, 3, 3, 384, 640, True),
+    (1, 8, 2, 300, 300, True), (1, 8, 2, 300, 700, False), (2, 32, 8, 1024, 1024, True),
+    (1, 32, 4, 640, 640, True), (1, 6, 2, 130, 130, True), (1, 5, 5, 1, 1, False),
+    (3, 4, 4, 129, 1000, True), (1, 16, 16, 16384, 16384, True),
+]
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,causal", CASES)
+def test_plan_covers_every_tile_once(B, Hq, Hkv, Sq, Sk, causal):
+    plan = lib.attn_plan(B, Hq, Hkv, Sq, Sk, 128, causal, 148)
+    g = Hq // Hkv
+    assert plan["pair_heads"] == (1 if g % 2 == 0 else 0)
+    assert plan["n_q_tiles"] == math.ceil(Sq / TILE) and plan["n_kv_blocks"] == math.ceil(Sk / TILE)
+    assert plan["ctas"] == min(148, plan["n_work"])
+    seen = {}
+    n_work = plan["n_work"]
+    step = 1 if n_work <= 4096 else 7  # large cases: a stride-7 sample plus the ends
+    ws = sorted(set(list(range(0, n_work, step)) + [n_work - 1]))
+    for w in ws:
+        it = lib.attn_plan_item(B, Hq, Hkv, Sq, Sk, 128, causal, w)
+        assert 0 <= it["b"] < B and 0 <= it["hkv"] < Hkv
+        for s in (0, 1):
+            hq, row0, n = it[f"hq{s}"], it[f"row0_{s}"], it[f"n_blocks_{s}"]
+            assert 0 <= hq < Hq and hq // g == it["hkv"] and row0 % TILE == 0
+            if row0 >= Sq:
+                assert n == 0
+                continue
+            assert n == visible_blocks_brute(row0, Sq, Sk, causal)
+            key = (it["b"], hq, row0)
+            assert key not in seen
+            seen[key] = w
+    if step == 1:
+        assert len(seen) == B * Hq * math.ceil(Sq / TILE)
+
+
+def test_causal_items_run_longest_first_inside_a_head():
+    B, H, S = 1, 2, 2048
+    plan = lib.attn_plan(B, H, H, S, S, 128, True, 148)
+    per = plan["items_per_group"]
+    cost = [sum(lib.attn_plan_item(B, H, H, S, S, 128, True, w)[f"n_blocks_{s}"] for s in (0, 1))
+            for w in range(plan["n_work"])]
+    for h in range(B * H):
+        c = cost[h * per:(h + 1) * per]
+        assert c == sorted(c, reverse=True)
+
+
+def test_scheduler_option_changes_grid_only():
+    lib.attn_set_option("scheduler", 0)
+    try:
+        plan = lib.attn_plan(2, 16, 16, 16384, 16384, 128, False, 148)
+        assert plan["ctas"] == plan["n_work"] == 2 * 16 * 64
+        lib.attn_set_option("scheduler", 1)
+        lib.attn_set_option("max_ctas", 100)
+        assert lib.attn_plan(2, 16, 16, 16384, 16384, 128, False, 148)["ctas"] == 100
+    finally:
+        lib.attn_set_option("scheduler", 2)
+        lib.attn_set_option("max_ctas", 0)
+
+
+def test_plan_rejects_bad_problems():
+    with pytest.raises(lib.AttnError):
+        lib.attn_plan(1, 3, 2, 128, 128, 128, False, 148)
+    with pytest.raises(lib.AttnError):
+        lib.attn_plan(1, 2, 2, 256, 128, 128, True, 148)
+    with pytest.raises(lib.AttnError):
+        lib.attn_plan_item(1, 2, 2, 128, 128, 128, False, 99)
