@@ -1,0 +1,310 @@
+#!/usr/bin/env python
+"""Benchmark of the fused attention forward pass (BF16, head dim 128) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole forward path (one `attn_fwd` call) over one batch of synthetic
+BF16 Q/K/V resident in HBM.  The default workload is the one the headline metric is quoted on:
+non-causal multi-head attention, 16 heads, 32768 tokens as 2 sequences of 16384.  The metric is
+TFLOP/s with 4*B*Hq*Sq*Sk*D FLOPs per call (halved when causal).
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs an independent
+replica of the same workload -- attention rows never cross (batch, head), so nothing is
+exchanged -- and the reported value is the sum over ranks divided by the slowest rank's time.
+
+`--impl reference` times the CPU fp64 oracle instead (rank 0 only), on a bounded sample of the
+same workload's rows per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from workloads import all_workloads, bf16_bits, make_workload_inputs  # noqa: E402
+
+METRIC = "attn_fwd_bf16_d128_tflops"
+UNIT = "TFLOP/s"
+DEFAULT_WORKLOAD = "mha_noncausal_s16384"
+FALLBACK_BF16_TFLOPS = 1590.0  # earlier measurement on this machine, used only without MEASURED_PEAKS.json
+NOMINAL_BF16_TFLOPS = 2250.0
+REFERENCE_ROWS_PER_STEP = 1024
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target oracle time of the cpu_baseline leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["bf16_tflops"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured"
+    return FALLBACK_BF16_TFLOPS, 1400.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, power, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+                power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        try:
+            os.unlink(self.file.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power))
+        return out
+
+
+def oracle_sample_tflops(w, q, k, v, n_rows, seed):
+    """Times the CPU oracle, as it stands, on `n_rows` seeded rows of the workload."""
+    from oracle import attn_oracle as orc
+    rng = np.random.default_rng(seed)  # uniform over (b, hq, i): unbiased under the causal mask
+    rows = np.stack([rng.integers(w.B, size=n_rows), rng.integers(w.Hq, size=n_rows),
+                     rng.integers(w.Sq, size=n_rows)], axis=1).astype(np.int32)
+    qb, kb, vb = bf16_bits(q), bf16_bits(k), bf16_bits(v)
+    t0 = time.perf_counter()
+    orc.attention_rows(qb, kb, vb, w.causal, w.scale, rows)
+    dt = time.perf_counter() - t0
+    # FLOPs of these rows under the metric's convention: 4 * Sk * D per (row), halved when causal
+    flops = len(rows) * 4.0 * w.Sk * w.D * (0.5 if w.causal else 1.0)
+    return flops / dt / 1e12, dt, len(rows), orc.default_threads()
+
+
+def run_reference(args, w):
+    """The oracle on host cores; each step is a bounded row sample of the workload."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    from oracle import attn_oracle as orc
+    orc.build()
+    q, k, v = make_workload_inputs(w)
+    for i in range(args.warmup):
+        oracle_sample_tflops(w, q, k, v, 64, seed=100 + i)
+    times, rows_done = [], 0
+    for i in range(args.steps):
+        _, dt, n, cores = oracle_sample_tflops(w, q, k, v, REFERENCE_ROWS_PER_STEP, seed=1000 + i)
+        times.append(dt)
+        rows_done += n
+    total = sum(times)
+    flops = rows_done * 4.0 * w.Sk * w.D * (0.5 if w.causal else 1.0)
+    value = flops / total / 1e12
+    sample = f"{REFERENCE_ROWS_PER_STEP} seeded query rows (all keys) of {w.name} per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "Sq": w.Sq, "Sk": w.Sk, "D": w.D,
+                   "causal": w.causal, "note": "CPU fp64 oracle on host cores, bounded row sample per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.default_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w):
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    import paper_2603_24517_b200 as lib
+    from paper_2603_24517_b200 import build as lib_build
+    lib_build.build()
+    lib.load_library()
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=dev)
+
+    # every rank: an independent replica of the workload (same shapes, rank-specific seed)
+    import dataclasses
+    w_rank = dataclasses.replace(w, seed=w.seed + 10007 * rank)
+    q_h, k_h, v_h = make_workload_inputs(w_rank)
+    q, k, v = q_h.to(dev), k_h.to(dev), v_h.to(dev)
+    o = torch.empty_like(q)
+    lse = torch.empty((w.B, w.Hq, w.Sq), dtype=torch.float32, device=dev)
+    scale = w.scale
+
+    def barrier():
+        if use_dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        lib.attn_fwd(q, k, v, o, lse, w.causal, scale)
+    barrier()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        lib.attn_fwd(q, k, v, o, lse, w.causal, scale)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    st, code, detail = lib.attn_last_device_status()
+    if st != 0:
+        raise SystemExit(f"device status {st} code {code:#x} detail {detail}")
+
+    # end to end through the host-buffer entry point: H2D of Q, K, V and D2H of O, LSE every step
+    qp, kp, vp = q_h.pin_memory(), k_h.pin_memory(), v_h.pin_memory()
+    op = torch.empty_like(q_h).pin_memory()
+    lp = torch.empty((w.B, w.Hq, w.Sq), dtype=torch.float32).pin_memory()
+    lib.attn_fwd_host(qp, kp, vp, op, lp, w.causal, scale, device=local)  # warm-up: allocates staging
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    for _ in range(args.e2e_steps):
+        lib.attn_fwd_host(qp, kp, vp, op, lp, w.causal, scale, device=local)
+    e3.record()
+    barrier()
+    ms_e2e = e2.elapsed_time(e3)
+    h2d = qp.numel() * 2 + kp.numel() * 2 + vp.numel() * 2
+    d2h = op.numel() * 2 + lp.numel() * 4
+    lib.attn_release_host_staging()
+
+    if use_dist:
+        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = float(t[0]), float(t[1])
+
+    if rank == 0:
+        ms_step = ms_total / args.steps
+        value = world * w.flops / (ms_step * 1e-3) / 1e12
+        e2e_value = world * w.flops / (ms_e2e / args.e2e_steps * 1e-3) / 1e12
+        peak_burst, peak_sustained, peak_kind = measured_peaks()
+        achieved = w.flops / (ms_step * 1e-3) / 1e12  # one GPU's kernel: one launch per step
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "Sq": w.Sq, "Sk": w.Sk,
+                       "D": w.D, "causal": w.causal, "parallelism": f"replicas x{world}",
+                       "l2": f"inputs+outputs {w.algorithmic_bytes / 2**20:.0f} MiB exceed the 126 MB L2; no flush",
+                       "flops_per_step": w.flops},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": args.e2e_steps},
+            "gpu_launches": args.steps,
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak_burst, "unit": UNIT,
+                         "frac": achieved / peak_burst, "peak_kind": f"{peak_kind} cuBLAS bf16 burst",
+                         "frac_of_sustained": achieved / peak_sustained,
+                         "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
+                         "traffic": TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": w.algorithmic_bytes},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            from oracle import attn_oracle as orc
+            orc.build()
+            rate, dt, n, cores = oracle_sample_tflops(w, q_h, k_h, v_h, 256, seed=1)
+            n_rows = int(max(256, min(200000, args.cpu_seconds * n / dt)))
+            rate, dt, n, cores = oracle_sample_tflops(w, q_h, k_h, v_h, n_rows, seed=2)
+            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": f"{n} seeded query rows (all keys) of {w.name}, {dt:.1f} s"}
+        print(json.dumps(line), flush=True)
+    if use_dist:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
+# profiles/ (None until a capture of the current kernel exists).
+TRAFFIC_BYTES: dict[str, float | None] = {}
+
+
+def main():
+    args = parse_args()
+    workloads = all_workloads()
+    if args.workload not in workloads:
+        raise SystemExit(f"unknown workload {args.workload}; choose from {sorted(workloads)}")
+    w = workloads[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
