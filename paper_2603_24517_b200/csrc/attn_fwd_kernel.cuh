@@ -182,30 +182,43 @@ __device__ __forceinline__ int consumer_next_work(const FwdParams& p, const Barr
 }
 
 // ------------------------------------------------------------------------------------------
-// MMA issue helpers (one thread)
+// MMA issue helpers.  The whole MMA warp runs the control flow, so that descriptors and tensor
+// memory addresses are warp-uniform values; only the elected lane issues the instructions.
 // ------------------------------------------------------------------------------------------
 constexpr uint32_t kIdescQK = make_idesc_bf16(kTile, kTile, 0, 0);     // A = Q, B = K, both K-major
 constexpr uint32_t kIdescPV = make_idesc_bf16(kTile, kHeadDim, 0, 1);  // A = P (tmem), B = V MN-major
 
+// Descriptor of a K-major [128 rows][128 head-dim] tile (Q or K) and of an MN-major V tile.
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t smem_addr) { return make_smem_desc_sw128(smem_addr, 16, 1024); }
+__device__ __forceinline__ uint64_t vtile_desc(uint32_t smem_addr) {
+  return make_smem_desc_sw128(smem_addr, kHalfBytes, 1024);
+}
+// The start-address field counts 16-byte units and never carries out of its 14 bits here
+// (shared memory addresses stay below 256 KB), so advancing a descriptor is one addition.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) { return desc + (bytes >> 4); }
+
 // S[128 x 128] = Q[128 x 128] K[128 x 128]^T : 8 steps of 16 along the head dimension.  A half
 // tile holds 64 head-dim elements per row (one 128-byte swizzle row), so a step advances 32 bytes
 // inside the half tile and the second half tile starts 16 KB later.
-__device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint32_t q_smem, uint32_t k_smem) {
+__device__ __forceinline__ void issue_qk(bool leader, uint32_t tmem_s, uint64_t q_desc, uint64_t k_desc) {
+  if (leader) {
 #pragma unroll
-  for (int kk = 0; kk < 8; ++kk) {
-    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-    mma_ss(tmem_s, make_smem_desc_sw128(q_smem + off, 16, 1024), make_smem_desc_sw128(k_smem + off, 16, 1024),
-           kIdescQK, kk > 0);
+    for (int kk = 0; kk < 8; ++kk) {
+      const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+      mma_ss(tmem_s, desc_advance(q_desc, off), desc_advance(k_desc, off), kIdescQK, kk > 0);
+    }
   }
 }
 // O[128 x 128] (+)= P[128 x 128 keys] V[128 keys x 128] : 8 steps of 16 keys.  P: 8 tensor-memory
 // columns per step (two BF16 per column).  V is MN-major: a key is one 128-byte row of a half
 // tile, 16 keys are 2048 bytes, the second 64 head-dim elements sit 16 KB later (leading offset).
-__device__ __forceinline__ void issue_pv(uint32_t tmem_o, uint32_t tmem_p, uint32_t v_smem, bool accumulate) {
+__device__ __forceinline__ void issue_pv(bool leader, uint32_t tmem_o, uint32_t tmem_p, uint64_t v_desc,
+                                         bool accumulate) {
+  if (leader) {
 #pragma unroll
-  for (int kk = 0; kk < 8; ++kk) {
-    mma_ts(tmem_o, tmem_p + kk * 8, make_smem_desc_sw128(v_smem + kk * 2048, kHalfBytes, 1024), kIdescPV,
-           (accumulate || kk > 0) ? 1u : 0u);
+    for (int kk = 0; kk < 8; ++kk) {
+      mma_ts(tmem_o, tmem_p + kk * 8, desc_advance(v_desc, kk * 2048), kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
+    }
   }
 }
 
@@ -267,32 +280,40 @@ __device__ __forceinline__ void role_loader(const FwdParams& p, const Barriers& 
   }
 }
 
+// Bounded wait by a whole warp with a warp-uniform result.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, WaitCtx ctx, int code) {
+  const bool ok = mbar_wait(bar, parity, ctx, code);
+  return __all_sync(0xffffffffu, ok);
+}
+
 __device__ __forceinline__ void role_mma(const FwdParams& p, const Barriers& bars, uint8_t* smem,
-                                         const volatile int* sched_w, WaitCtx ctx, uint32_t tmem) {
+                                         const volatile int* sched_w, WaitCtx ctx, uint32_t tmem, int lane) {
+  const bool leader = elect_one();
   const uint32_t smem_base = smem_u32(smem);
+  const uint64_t q_desc[2] = {kmajor_desc(smem_base + kSmemQ), kmajor_desc(smem_base + kSmemQ + kTileBytes)};
   uint32_t kv_cnt = 0;
   uint32_t q_cnt[2] = {0, 0};   // per-stage work items seen (phase of q_full / o_empty)
   uint32_t sp_cnt[2] = {0, 0};  // per-stage K/V blocks seen (phase of p_full)
   for (int it = 0;; ++it) {
-    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleMma, true, false);
+    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleMma, lane == 0, true);
     if (w < 0 || w >= p.n_work) return;
     Work wk;
     decode_work(p, w, wk);
     // S_s(0) for both stages
     {
       const uint32_t slot = kv_cnt % kKvSlots, par = (kv_cnt / kKvSlots) & 1;
-      if (!mbar_wait(&bars.kv_full[slot], par, ctx, kRoleMma | kBarKvFull)) return;
-      const uint32_t k_smem = smem_base + kSmemKv + slot * kTileBytes;
+      if (!mbar_wait_warp(&bars.kv_full[slot], par, ctx, kRoleMma | kBarKvFull)) return;
+      const uint64_t k_desc = kmajor_desc(smem_base + kSmemKv + slot * kTileBytes);
 #pragma unroll
       for (int s = 0; s < 2; ++s) {
         if (wk.n[s] > 0) {
-          if (!mbar_wait(&bars.q_full[s], q_cnt[s] & 1, ctx, kRoleMma | kBarQFull)) return;
+          if (!mbar_wait_warp(&bars.q_full[s], q_cnt[s] & 1, ctx, kRoleMma | kBarQFull)) return;
           tc_fence_after_sync();
-          issue_qk(tmem + s * kTile, smem_base + kSmemQ + s * kTileBytes, k_smem);
-          mma_commit(&bars.s_full[s]);
+          issue_qk(leader, tmem + s * kTile, q_desc[s], k_desc);
+          if (leader) mma_commit(&bars.s_full[s]);
         }
       }
-      mma_commit(&bars.kv_empty[slot]);
+      if (leader) mma_commit(&bars.kv_empty[slot]);
       ++kv_cnt;
     }
     for (int j = 0; j < wk.nmax; ++j) {
@@ -305,34 +326,36 @@ __device__ __forceinline__ void role_mma(const FwdParams& p, const Barriers& bar
         kpar = (kv_cnt / kKvSlots) & 1;
         ++kv_cnt;
       }
-      if (!mbar_wait(&bars.kv_full[vslot], vpar, ctx, kRoleMma | kBarKvFull)) return;
+      if (!mbar_wait_warp(&bars.kv_full[vslot], vpar, ctx, kRoleMma | kBarKvFull)) return;
       bool k_ready = false;
-      const uint32_t v_smem = smem_base + kSmemKv + vslot * kTileBytes;
-      const uint32_t k_smem = smem_base + kSmemKv + kslot * kTileBytes;
+      const uint64_t v_desc = vtile_desc(smem_base + kSmemKv + vslot * kTileBytes);
+      const uint64_t k_desc = kmajor_desc(smem_base + kSmemKv + kslot * kTileBytes);
 #pragma unroll
       for (int s = 0; s < 2; ++s) {
         if (j < wk.n[s]) {
           if (j == 0) {  // the previous item's O_s must have left tensor memory
-            if (!mbar_wait(&bars.o_empty[s], (q_cnt[s] & 1) ^ 1, ctx, kRoleMma | kBarOEmpty)) return;
+            if (!mbar_wait_warp(&bars.o_empty[s], (q_cnt[s] & 1) ^ 1, ctx, kRoleMma | kBarOEmpty)) return;
           }
-          if (!mbar_wait(&bars.p_full[s], sp_cnt[s] & 1, ctx, kRoleMma | kBarPFull)) return;
+          if (!mbar_wait_warp(&bars.p_full[s], sp_cnt[s] & 1, ctx, kRoleMma | kBarPFull)) return;
           ++sp_cnt[s];
           tc_fence_after_sync();
-          issue_pv(tmem + 2 * kTile + s * kTile, tmem + s * kTile, v_smem, j > 0);
-          if (j == wk.n[s] - 1) mma_commit(&bars.o_full[s]);
+          issue_pv(leader, tmem + 2 * kTile + s * kTile, tmem + s * kTile, v_desc, j > 0);
+          if (leader && j == wk.n[s] - 1) mma_commit(&bars.o_full[s]);
           if (j + 1 < wk.n[s]) {
             if (!k_ready) {
-              if (!mbar_wait(&bars.kv_full[kslot], kpar, ctx, kRoleMma | kBarKvFull)) return;
+              if (!mbar_wait_warp(&bars.kv_full[kslot], kpar, ctx, kRoleMma | kBarKvFull)) return;
               tc_fence_after_sync();
               k_ready = true;
             }
-            issue_qk(tmem + s * kTile, smem_base + kSmemQ + s * kTileBytes, k_smem);
-            mma_commit(&bars.s_full[s]);
+            issue_qk(leader, tmem + s * kTile, q_desc[s], k_desc);
+            if (leader) mma_commit(&bars.s_full[s]);
           }
         }
       }
-      mma_commit(&bars.kv_empty[vslot]);
-      if (has_next) mma_commit(&bars.kv_empty[kslot]);
+      if (leader) {
+        mma_commit(&bars.kv_empty[vslot]);
+        if (has_next) mma_commit(&bars.kv_empty[kslot]);
+      }
     }
 #pragma unroll
     for (int s = 0; s < 2; ++s) {
@@ -607,7 +630,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   } else {
     reg_dealloc<ATTN_REGS_OTHER>();
     if (warp == 12) {
-      if (lane == 0) role_mma(p, bars, smem, sched_w, ctx, tmem);
+      role_mma(p, bars, smem, sched_w, ctx, tmem, lane);
     } else if (warp == 13) {
       if (lane == 0) {
         role_loader(p, bars, smem, sched_w, ctx, &tm_q, &tm_k, &tm_v);
