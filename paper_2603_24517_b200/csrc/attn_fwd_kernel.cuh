@@ -30,14 +30,19 @@ constexpr float kRescaleThreshold = 8.0f;  // log2 units a row maximum may lag b
 // Registers per thread of each role after the setmaxnreg re-split of the CTA's 64K registers:
 // 8 softmax warps, 4 epilogue warps, 4 other warps; 8 * a + 4 * b + 4 * c must not exceed 2048.
 #ifndef ATTN_REGS_SOFTMAX
-#define ATTN_REGS_SOFTMAX 176
+#define ATTN_REGS_SOFTMAX 192
 #endif
 #ifndef ATTN_REGS_EPILOGUE
-#define ATTN_REGS_EPILOGUE 80
+#define ATTN_REGS_EPILOGUE 64
 #endif
 #ifndef ATTN_REGS_OTHER
-#define ATTN_REGS_OTHER 80
+#define ATTN_REGS_OTHER 64
 #endif
+// Of every four column pairs of a score row, how many take the polynomial exp2 (0..4).
+#ifndef ATTN_EXP2_POLY_PAIRS
+#define ATTN_EXP2_POLY_PAIRS 1
+#endif
+constexpr int kExp2PolyPairs = ATTN_EXP2_POLY_PAIRS;
 static_assert(8 * ATTN_REGS_SOFTMAX + 4 * ATTN_REGS_EPILOGUE + 4 * ATTN_REGS_OTHER <= 2048, "register split");
 
 constexpr int kSmemQ = 0;
@@ -123,11 +128,19 @@ struct WaitCtx {
 };
 
 __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, WaitCtx ctx, int code) {
-  const uint64_t t0 = global_timer_ns();
+  // The clock is read only every kSpinsPerCheck failed polls: reading it costs more than a poll,
+  // and a waiter must notice the phase flip as soon as it happens.
+  constexpr int kSpinsPerCheck = 256;
+  uint64_t t0 = 0;
   for (;;) {
-    if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+    for (int i = 0; i < kSpinsPerCheck; ++i) {
+      if (mbar_try_wait(bar, parity)) return true;
+    }
     if (*ctx.abort_flag) return false;
-    if (global_timer_ns() - t0 > kWaitLimitNs) {
+    const uint64_t now = global_timer_ns();
+    if (t0 == 0) t0 = now;
+    if (now - t0 > kWaitLimitNs) {
       *ctx.abort_flag = 1;
       if (atomicCAS(ctx.status, 0, code) == 0) ctx.status[1] = static_cast<int>(blockIdx.x);
       return false;
@@ -441,28 +454,38 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
           }
         }
       }
+      // P = exp2(S * c - m_used * c) on pairs of columns with packed fp32 arithmetic.  Of every
+      // four pairs, kExp2PolyPairs are evaluated by the polynomial on the FMA pipe and the rest
+      // by the special-function unit, so that neither unit alone bounds the row.
       const float neg_mc = -m_used * c;
-      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+      const float2 c2 = make_float2(c, c);
+      const float2 nm2 = make_float2(neg_mc, neg_mc);
+      float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
         uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-          const float e0 = ex2_approx(fmaf(X(cc * 32 + i + 0), c, neg_mc));
-          const float e1 = ex2_approx(fmaf(X(cc * 32 + i + 1), c, neg_mc));
-          const float e2 = ex2_approx(fmaf(X(cc * 32 + i + 2), c, neg_mc));
-          const float e3 = ex2_approx(fmaf(X(cc * 32 + i + 3), c, neg_mc));
-          l0 += e0;
-          l1 += e1;
-          l2 += e2;
-          l3 += e3;
-          pk[i / 2] = pack_bf16x2(e0, e1);
-          pk[i / 2 + 1] = pack_bf16x2(e2, e3);
+        for (int pr = 0; pr < 16; ++pr) {
+          const int i = cc * 32 + pr * 2;
+          const float2 x = fma2(make_float2(X(i), X(i + 1)), c2, nm2);
+          float2 e;
+          if ((pr & 3) < kExp2PolyPairs) {
+            e = exp2_poly2(x);
+          } else {
+            e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+          }
+          if (pr & 1) {
+            lb = add2(lb, e);
+          } else {
+            la = add2(la, e);
+          }
+          pk[pr] = pack_bf16x2(e.x, e.y);
         }
         tmem_st_x16(t_s + cc * 16, pk);
       }
 #undef X
-      l += (l0 + l1) + (l2 + l3);
+      la = add2(la, lb);
+      l += la.x + la.y;
       tmem_wait_st();
       tc_fence_before_sync();
       if (lane == 0) mbar_arrive(&bars.p_full[s]);
