@@ -131,6 +131,22 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks of the default process group
+    (identity when torch.distributed is not initialised).  Works with nccl and gloo."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_tflops(flops_per_replica: float, world: int, ms_per_step: float) -> float:
+    """Throughput of `world` independent replicas that all finish a step within `ms_per_step`."""
+    return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
+
+
 def oracle_sample_tflops(w, q, k, v, n_rows, seed):
     """Times the CPU oracle, as it stands, on `n_rows` seeded rows of the workload."""
     from oracle import attn_oracle as orc
@@ -247,15 +263,12 @@ def run_ours(args, w):
     d2h = op.numel() * 2 + lp.numel() * 4
     lib.attn_release_host_staging()
 
-    if use_dist:
-        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], device=dev)
 
     if rank == 0:
         ms_step = ms_total / args.steps
-        value = world * w.flops / (ms_step * 1e-3) / 1e12
-        e2e_value = world * w.flops / (ms_e2e / args.e2e_steps * 1e-3) / 1e12
+        value = whole_job_tflops(w.flops, world, ms_step)
+        e2e_value = whole_job_tflops(w.flops, world, ms_e2e / args.e2e_steps)
         peak_burst, peak_sustained, peak_kind = measured_peaks()
         achieved = w.flops / (ms_step * 1e-3) / 1e12  # one GPU's kernel: one launch per step
         line = {
