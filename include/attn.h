@@ -32,7 +32,8 @@ typedef enum {
   ATTN_ERR_ALIGN = 4,       /* q, k, v or o not 16-byte aligned; lse not 4-byte aligned */
   ATTN_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed (descriptor, launch, copy) */
   ATTN_ERR_ARCH = 6,        /* the current device is not compute capability 10.x */
-  ATTN_ERR_TIMEOUT = 7      /* a bounded wait inside a kernel expired (see attn_last_device_status) */
+  ATTN_ERR_TIMEOUT = 7,     /* a bounded wait inside a kernel expired (see attn_last_device_status) */
+  ATTN_ERR_TOO_LARGE = 8    /* attn_fwd_noalloc only: the problem exceeds ATTN_NOALLOC_MAX_Q_TILES */
 } attn_status_t;
 
 /*
@@ -78,6 +79,38 @@ attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, flo
 attn_status_t attn_fwd_host(const void* q, const void* k, const void* v, void* o, float* lse,
                             int B, int Hq, int Hkv, int Sq, int Sk, int D,
                             int causal, float scale, void* stream);
+
+/*
+ * attn_fwd_noalloc -- attn_fwd for callers that must not allocate device memory.
+ * (The paper has no counterpart; this is a convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a memory budget that
+ * was handed out in full at start-up (an inference server that pre-reserves all of HBM for
+ * its own pools), on a latency-critical thread that may not take the driver's allocation
+ * lock, or in an embedding runtime that forbids library-side allocations altogether.
+ * attn_fwd allocates a few KB of scheduler state with cudaMalloc on its first call per
+ * device; this entry point never calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ * Same arguments, layouts, arithmetic and results as attn_fwd (device pointers, asynchronous
+ * on `stream`).  The kernel's scratch -- the tile scheduler's work counter and the status
+ * words of its bounded waits -- lives in a 256-byte array that is part of the library image,
+ * so every GPU that loads the library carries those 256 bytes until the process exits.
+ *
+ * Limits and rules:
+ *   - B * Hq * ceil(Sq / 128) must not exceed ATTN_NOALLOC_MAX_Q_TILES, else
+ *     ATTN_ERR_TOO_LARGE is returned and nothing is launched.
+ *   - All calls on a device share the one scratch array.  Each call clears the words that
+ *     must start at zero (on `stream`, before its kernel), so back-to-back calls on one
+ *     stream are fine; two calls whose kernels can overlap on the GPU (different streams,
+ *     no dependency) race on the work counter and give wrong results.  Use attn_fwd there.
+ *   - The first call on each device looks up the array's device address and sets the
+ *     kernel's shared-memory attribute; make that first call outside any stream capture.
+ *   - Expired bounded waits are recorded in the scratch array only; no API reads them back.
+ */
+#define ATTN_NOALLOC_MAX_Q_TILES (1 << 20)
+attn_status_t attn_fwd_noalloc(const void* q, const void* k, const void* v, void* o, float* lse,
+                               int B, int Hq, int Hkv, int Sq, int Sk, int D,
+                               int causal, float scale, void* stream);
 
 /* Releases the staging buffers attn_fwd_host holds on the current device. */
 attn_status_t attn_release_host_staging(void);

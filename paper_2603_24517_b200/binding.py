@@ -18,9 +18,9 @@ LIB_PATH = os.path.join(_PKG, "libattn_b200.so")
 ATTN_OK = 0
 STATUS_NAMES = {
     0: "ATTN_OK", 1: "ATTN_ERR_NULL", 2: "ATTN_ERR_SHAPE", 3: "ATTN_ERR_UNSUPPORTED", 4: "ATTN_ERR_ALIGN",
-    5: "ATTN_ERR_CUDA", 6: "ATTN_ERR_ARCH", 7: "ATTN_ERR_TIMEOUT",
+    5: "ATTN_ERR_CUDA", 6: "ATTN_ERR_ARCH", 7: "ATTN_ERR_TIMEOUT", 8: "ATTN_ERR_TOO_LARGE",
 }
-EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_host", "attn_release_host_staging", "attn_set_option",
+EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_host", "attn_fwd_noalloc", "attn_release_host_staging", "attn_set_option",
                     "attn_plan", "attn_plan_item", "attn_status_str", "attn_version",
                     "attn_last_device_status")
 
@@ -48,6 +48,8 @@ def load_library() -> ctypes.CDLL:
     lib.attn_fwd.restype = ci
     lib.attn_fwd_host.argtypes = fwd_args
     lib.attn_fwd_host.restype = ci
+    lib.attn_fwd_noalloc.argtypes = fwd_args
+    lib.attn_fwd_noalloc.restype = ci
     lib.attn_release_host_staging.argtypes = []
     lib.attn_release_host_staging.restype = ci
     lib.attn_set_option.argtypes = [ctypes.c_char_p, ci]
@@ -98,6 +100,28 @@ def attn_fwd(q, k, v, o, lse, causal: bool, scale: float, stream=None) -> None:
     st = attn_fwd_status(q, k, v, o, lse, causal, scale, stream)
     if st != ATTN_OK:
         raise AttnError(st, "attn_fwd")
+
+
+def attn_fwd_noalloc_status(q, k, v, o, lse, causal: bool, scale: float, stream=None) -> int:
+    """Calls ``attn_fwd_noalloc`` on CUDA tensors and returns its raw status code."""
+    B, Hq, Hkv, Sq, Sk, D = _check_layout(q, k, v, o, lse, "cuda")
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        return load_library().attn_fwd_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                               None if lse is None else lse.data_ptr(),
+                                               B, Hq, Hkv, Sq, Sk, D, int(bool(causal)), float(scale), stream)
+
+
+def attn_fwd_noalloc(q, k, v, o, lse, causal: bool, scale: float, stream=None) -> None:
+    """``attn_fwd_noalloc`` of the C ABI: ``attn_fwd`` for callers that may not allocate device
+    memory.  The library keeps the kernel's scratch in a fixed 256-byte device array instead
+    of allocating it, so calls that could overlap on the GPU must not use this entry point,
+    and problems beyond ``ATTN_NOALLOC_MAX_Q_TILES`` query tiles are refused
+    (``ATTN_ERR_TOO_LARGE``).  Make the first call on a device outside stream capture."""
+    st = attn_fwd_noalloc_status(q, k, v, o, lse, causal, scale, stream)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_fwd_noalloc")
 
 
 def attn_fwd_host(q, k, v, o, lse, causal: bool, scale: float, device=0, stream=None) -> None:

@@ -250,6 +250,87 @@ attn_status_t attn_fwd_host(const void* q, const void* k, const void* v, void* o
   return cudaStreamSynchronize(s) == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
+// ------------------------------------------------------------------------------------------
+// attn_fwd_noalloc: the same kernel with its scratch in a static device array.
+// ------------------------------------------------------------------------------------------
+namespace {
+
+// Scratch of the no-allocation entry point, one copy per device that loads this library:
+// word 0 = tile scheduler work counter, words 2-3 = status of expired waits, the rest unused.
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device pointer.
+static __device__ __align__(256) unsigned int g_noalloc_scratch[64];
+
+struct NoAllocDevice {
+  bool ready = false;
+  int sm_count = 0;
+  unsigned int* scratch = nullptr;  // device address of g_noalloc_scratch on this device
+};
+NoAllocDevice g_noalloc_dev[kMaxDevices];
+
+// Once per device, with that device current: architecture check, TMA encoder lookup, kernel
+// attribute, and the device address of the scratch array.  Allocates nothing.
+attn_status_t noalloc_device(NoAllocDevice** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ATTN_ERR_CUDA;
+  NoAllocDevice& d = g_noalloc_dev[dev];
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!d.ready) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ATTN_ERR_CUDA;
+    if (major != 10) return ATTN_ERR_ARCH;
+    if (g_encode == nullptr) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+          fn == nullptr)
+        return ATTN_ERR_CUDA;
+      g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    void* ptr = nullptr;
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaFuncSetAttribute(attn::attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             attn::kSmemBytes) != cudaSuccess ||
+        cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr)
+      return ATTN_ERR_CUDA;
+    d.scratch = static_cast<unsigned int*>(ptr);
+    d.ready = true;
+  }
+  *out = &d;
+  return ATTN_OK;
+}
+
+}  // namespace
+
+attn_status_t attn_fwd_noalloc(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq,
+                               int Hkv, int Sq, int Sk, int D, int causal, float scale, void* stream) {
+  attn_status_t st = check_args(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, scale, true);
+  if (st != ATTN_OK) return st;
+  if (static_cast<long long>(B) * Hq * ((Sq + attn::kTile - 1) / attn::kTile) > ATTN_NOALLOC_MAX_Q_TILES)
+    return ATTN_ERR_TOO_LARGE;
+  NoAllocDevice* dev = nullptr;
+  st = noalloc_device(&dev);
+  if (st != ATTN_OK) return st;
+
+  CUtensorMap tm_q, tm_k, tm_v, tm_o;
+  if (!make_tensor_map(&tm_q, q, B, Sq, Hq) || !make_tensor_map(&tm_k, k, B, Sk, Hkv) ||
+      !make_tensor_map(&tm_v, v, B, Sk, Hkv) || !make_tensor_map(&tm_o, o, B, Sq, Hq))
+    return ATTN_ERR_CUDA;
+
+  FwdParams p;
+  fill_plan(&p, B, Hq, Hkv, Sq, Sk, causal);
+  p.scale = scale;
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.lse = lse;
+  p.counter = dev->scratch;                               // word 0
+  p.status = reinterpret_cast<int*>(dev->scratch + 2);    // words 2-3
+  const int grid = plan_grid(p, dev->sm_count);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // the array keeps the previous call's contents: counter and status must start at zero
+  if (cudaMemsetAsync(dev->scratch, 0, 4 * sizeof(unsigned int), s) != cudaSuccess) return ATTN_ERR_CUDA;
+  attn::attn_fwd_kernel<<<grid, attn::kThreads, attn::kSmemBytes, s>>>(tm_q, tm_k, tm_v, tm_o, p);
+  return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
 attn_status_t attn_release_host_staging(void) {
   int devid = 0;
   if (cudaGetDevice(&devid) != cudaSuccess || devid < 0 || devid >= kMaxDevices) return ATTN_ERR_CUDA;
@@ -287,6 +368,7 @@ const char* attn_status_str(attn_status_t status) {
     case ATTN_ERR_CUDA: return "ATTN_ERR_CUDA";
     case ATTN_ERR_ARCH: return "ATTN_ERR_ARCH";
     case ATTN_ERR_TIMEOUT: return "ATTN_ERR_TIMEOUT";
+    case ATTN_ERR_TOO_LARGE: return "ATTN_ERR_TOO_LARGE";
   }
   return "ATTN_ERR_UNKNOWN";
 }
