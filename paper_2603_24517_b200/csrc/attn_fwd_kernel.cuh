@@ -49,7 +49,7 @@ constexpr int kSmemQ = 0;
 constexpr int kSmemKv = 2 * kTileBytes;
 constexpr int kSmemStats = kSmemKv + kKvSlots * kTileBytes;  // float [2 stages][2][128]
 constexpr int kSmemBars = kSmemStats + 2 * 2 * kTile * 4;
-constexpr int kNumBars = 2 + 2 + 2 * kKvSlots + 2 * 9;
+constexpr int kNumBars = 2 + 2 + 2 * kKvSlots + 2 * 10;
 constexpr int kSmemMisc = kSmemBars + kNumBars * 8;  // tmem base, abort flag, sched slots
 constexpr int kSmemBytes = kSmemMisc + 32;
 
@@ -156,7 +156,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, WaitCt
 enum : int {
   kRoleLoad = 1 << 8, kRoleMma = 2 << 8, kRoleSoftmax = 3 << 8, kRoleEpilogue = 4 << 8,
   kBarQFull = 1, kBarQEmpty = 2, kBarKvFull = 3, kBarKvEmpty = 4, kBarSFull = 5, kBarPFull = 6,
-  kBarOFull = 7, kBarOEmpty = 8, kBarLFull = 9, kBarLEmpty = 10, kBarSchedFull = 11, kBarSchedEmpty = 12, kBarStFull = 13,
+  kBarOFull = 7, kBarOEmpty = 8, kBarLFull = 9, kBarLEmpty = 10, kBarSchedFull = 11, kBarSchedEmpty = 12, kBarStFull = 13, kBarPHalf = 14,
   kBadSmemAlign = 0x7001
 };
 
@@ -166,7 +166,8 @@ struct Barriers {
   uint64_t* kv_full;   // [kKvSlots]
   uint64_t* kv_empty;  // [kKvSlots]  MMA commit -> loader
   uint64_t* s_full;    // [2]  MMA commit -> softmax
-  uint64_t* p_full;    // [2]  softmax (4 warps) -> MMA
+  uint64_t* p_half;    // [2]  softmax (4 warps): first 64 keys of P written -> MMA
+  uint64_t* p_full;    // [2]  softmax (4 warps): all of P written -> MMA
   uint64_t* o_full;    // [2]  MMA commit (last P V) -> epilogue
   uint64_t* o_empty;   // [2]  epilogue (4 warps) -> MMA
   uint64_t* l_full;    // [2]  softmax (128 threads) -> epilogue
@@ -226,11 +227,14 @@ __device__ __forceinline__ void issue_qk(bool leader, uint32_t tmem_s, uint64_t 
 // columns per step (two BF16 per column).  V is MN-major: a key is one 128-byte row of a half
 // tile, 16 keys are 2048 bytes, the second 64 head-dim elements sit 16 KB later (leading offset).
 __device__ __forceinline__ void issue_pv(bool leader, uint32_t tmem_o, uint32_t tmem_p, uint64_t v_desc,
-                                         bool accumulate) {
+                                         bool accumulate, int kk_begin, int kk_end) {
   if (leader) {
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk) {
-      mma_ts(tmem_o, tmem_p + kk * 8, desc_advance(v_desc, kk * 2048), kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
+      if (kk >= kk_begin && kk < kk_end) {
+        mma_ts(tmem_o, tmem_p + kk * 8, desc_advance(v_desc, kk * 2048), kIdescPV,
+               (accumulate || kk > 0) ? 1u : 0u);
+      }
     }
   }
 }
@@ -349,10 +353,15 @@ __device__ __forceinline__ void role_mma(const FwdParams& p, const Barriers& bar
           if (j == 0) {  // the previous item's O_s must have left tensor memory
             if (!mbar_wait_warp(&bars.o_empty[s], (q_cnt[s] & 1) ^ 1, ctx, kRoleMma | kBarOEmpty)) return;
           }
+          // P arrives in two halves of 64 keys: the first half of P V runs while the softmax
+          // warps are still exponentiating the second half
+          if (!mbar_wait_warp(&bars.p_half[s], sp_cnt[s] & 1, ctx, kRoleMma | kBarPHalf)) return;
+          tc_fence_after_sync();
+          issue_pv(leader, tmem + 2 * kTile + s * kTile, tmem + s * kTile, v_desc, j > 0, 0, 4);
           if (!mbar_wait_warp(&bars.p_full[s], sp_cnt[s] & 1, ctx, kRoleMma | kBarPFull)) return;
           ++sp_cnt[s];
           tc_fence_after_sync();
-          issue_pv(leader, tmem + 2 * kTile + s * kTile, tmem + s * kTile, v_desc, j > 0);
+          issue_pv(leader, tmem + 2 * kTile + s * kTile, tmem + s * kTile, v_desc, j > 0, 4, 8);
           if (leader && j == wk.n[s] - 1) mma_commit(&bars.o_full[s]);
           if (j + 1 < wk.n[s]) {
             if (!k_ready) {
@@ -482,6 +491,11 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
           pk[pr] = pack_bf16x2(e.x, e.y);
         }
         tmem_st_x16(t_s + cc * 16, pk);
+        if (cc == 1) {  // the first 64 keys of P are in tensor memory
+          tmem_wait_st();
+          tc_fence_before_sync();
+          if (lane == 0) mbar_arrive(&bars.p_half[s]);
+        }
       }
 #undef X
       la = add2(la, lb);
@@ -586,7 +600,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   bars.kv_full = bars.q_empty + 2;
   bars.kv_empty = bars.kv_full + kKvSlots;
   bars.s_full = bars.kv_empty + kKvSlots;
-  bars.p_full = bars.s_full + 2;
+  bars.p_half = bars.s_full + 2;
+  bars.p_full = bars.p_half + 2;
   bars.o_full = bars.p_full + 2;
   bars.o_empty = bars.o_full + 2;
   bars.l_full = bars.o_empty + 2;
@@ -612,6 +627,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(&bars.q_full[i], 1);
       mbar_init(&bars.q_empty[i], 1);
       mbar_init(&bars.s_full[i], 1);
+      mbar_init(&bars.p_half[i], 4);
       mbar_init(&bars.p_full[i], 4);
       mbar_init(&bars.o_full[i], 1);
       mbar_init(&bars.o_empty[i], 4);
