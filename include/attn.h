@@ -122,6 +122,10 @@ attn_status_t attn_release_host_staging(void);
  *                 1 = persistent CTAs, static round-robin over work items
  *                 2 = persistent CTAs, dynamic work counter (default)
  *   "max_ctas"    0 = one per SM (default), else an upper bound on persistent CTAs
+ *   "kernel"      0 = dual query stage: a CTA runs two 128-row query tiles against one stream
+ *                     of K/V tiles, one score buffer each (default)
+ *                 1 = triple score buffer: a CTA runs one query tile with three score tiles
+ *                     in flight and two softmax groups that alternate K/V blocks
  */
 attn_status_t attn_set_option(const char* name, int value);
 
@@ -139,7 +143,8 @@ attn_status_t attn_set_option(const char* name, int value);
  *
  * attn_plan_item fills item[0..7] = { b, hkv, hq0, hq1, row0_0, row0_1, n_blocks_0,
  * n_blocks_1 } for work item `w` in launch order (causal: longest items first inside each
- * head).  n_blocks_s = 0 marks an unused stage (its rows lie beyond Sq).
+ * head).  n_blocks_s = 0 marks an unused stage (its rows lie beyond Sq; with "kernel" = 1
+ * every item has one tile and stage 1 is always unused).
  * Both return ATTN_ERR_SHAPE / ATTN_ERR_UNSUPPORTED like attn_fwd, ATTN_ERR_SHAPE for w
  * out of range.
  */

@@ -7,6 +7,7 @@
 
 #include "../../include/attn.h"
 #include "attn_fwd_kernel.cuh"
+#include "attn_fwd_sb3.cuh"
 
 namespace {
 
@@ -36,6 +37,7 @@ DeviceState g_dev[kMaxDevices];
 EncodeTiledFn g_encode = nullptr;
 std::atomic<int> g_opt_scheduler{2};
 std::atomic<int> g_opt_max_ctas{0};
+std::atomic<int> g_opt_kernel{0};  // 0: dual query stage, 1: triple score buffer
 
 // Per-device one-time set-up: architecture check, kernel attribute, scheduler counters and
 // status word.  Returns the state or nullptr (with *st set).
@@ -75,6 +77,8 @@ DeviceState* device_state(attn_status_t* st) {
   if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
       cudaFuncSetAttribute(attn::attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            attn::kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(attn::sb3::attn_fwd_sb3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           attn::sb3::kSmemBytes3) != cudaSuccess ||
       cudaMalloc(&d.counters, kCounterSlots * sizeof(unsigned int)) != cudaSuccess ||
       cudaMalloc(&d.status, 2 * sizeof(int)) != cudaSuccess ||
       cudaMemset(d.status, 0, 2 * sizeof(int)) != cudaSuccess) {
@@ -129,15 +133,33 @@ void fill_plan(FwdParams* p, int B, int Hq, int Hkv, int Sq, int Sk, int causal)
   p->off = Sk - Sq;
   p->n_qt = (Sq + attn::kTile - 1) / attn::kTile;
   p->n_kb = (Sk + attn::kTile - 1) / attn::kTile;
-  p->pair_heads = (p->group % 2 == 0) ? 1 : 0;
-  if (p->pair_heads) {
-    p->items_per_group = p->n_qt * (p->group / 2);
-    p->n_work = B * Hkv * p->items_per_group;
+  p->kernel = g_opt_kernel.load();
+  if (p->kernel == 1) {  // triple score buffer: one query tile per work item
+    p->pair_heads = 0;
+    p->items_per_group = p->n_qt;
+    p->n_work = B * Hq * p->n_qt;
   } else {
-    p->items_per_group = (p->n_qt + 1) / 2;
-    p->n_work = B * Hq * p->items_per_group;
+    p->pair_heads = (p->group % 2 == 0) ? 1 : 0;
+    if (p->pair_heads) {
+      p->items_per_group = p->n_qt * (p->group / 2);
+      p->n_work = B * Hkv * p->items_per_group;
+    } else {
+      p->items_per_group = (p->n_qt + 1) / 2;
+      p->n_work = B * Hq * p->items_per_group;
+    }
   }
   p->dynamic = (g_opt_scheduler.load() == 2) ? 1 : 0;
+}
+
+// Launches the kernel selected by the "kernel" option (the plan in `p` was made for it).
+cudaError_t launch_fwd(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                       const CUtensorMap& tm_o, const FwdParams& p, int grid, cudaStream_t s) {
+  if (p.kernel == 1) {
+    attn::sb3::attn_fwd_sb3_kernel<<<grid, attn::kThreads, attn::sb3::kSmemBytes3, s>>>(tm_q, tm_k, tm_v, tm_o, p);
+  } else {
+    attn::attn_fwd_kernel<<<grid, attn::kThreads, attn::kSmemBytes, s>>>(tm_q, tm_k, tm_v, tm_o, p);
+  }
+  return cudaGetLastError();
 }
 
 int plan_grid(const FwdParams& p, int sm_count) {
@@ -180,6 +202,13 @@ attn_status_t attn_plan_item(int B, int Hq, int Hkv, int Sq, int Sk, int D, int 
   FwdParams p;
   fill_plan(&p, B, Hq, Hkv, Sq, Sk, causal);
   if (w < 0 || w >= p.n_work) return ATTN_ERR_SHAPE;
+  if (p.kernel == 1) {  // one tile per item: the second stage is reported as unused
+    attn::sb3::Item it;
+    attn::sb3::decode_item(p, w, it);
+    item[0] = it.b; item[1] = it.hkv; item[2] = it.hq; item[3] = it.hq;
+    item[4] = it.row0; item[5] = p.n_qt * attn::kTile; item[6] = it.n; item[7] = 0;
+    return ATTN_OK;
+  }
   attn::Work wk;
   attn::decode_work(p, w, wk);
   item[0] = wk.b; item[1] = wk.hkv; item[2] = wk.hq[0]; item[3] = wk.hq[1];
@@ -212,8 +241,7 @@ attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, flo
     p.counter = dev->counters + slot;
     if (cudaMemsetAsync(p.counter, 0, sizeof(unsigned int), s) != cudaSuccess) return ATTN_ERR_CUDA;
   }
-  attn::attn_fwd_kernel<<<grid, attn::kThreads, attn::kSmemBytes, s>>>(tm_q, tm_k, tm_v, tm_o, p);
-  return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+  return launch_fwd(tm_q, tm_k, tm_v, tm_o, p, grid, s) == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
 attn_status_t attn_fwd_host(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq,
@@ -290,6 +318,8 @@ attn_status_t noalloc_device(NoAllocDevice** out) {
     if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaFuncSetAttribute(attn::attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              attn::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(attn::sb3::attn_fwd_sb3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             attn::sb3::kSmemBytes3) != cudaSuccess ||
         cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr)
       return ATTN_ERR_CUDA;
     d.scratch = static_cast<unsigned int*>(ptr);
@@ -327,8 +357,7 @@ attn_status_t attn_fwd_noalloc(const void* q, const void* k, const void* v, void
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // the array keeps the previous call's contents: counter and status must start at zero
   if (cudaMemsetAsync(dev->scratch, 0, 4 * sizeof(unsigned int), s) != cudaSuccess) return ATTN_ERR_CUDA;
-  attn::attn_fwd_kernel<<<grid, attn::kThreads, attn::kSmemBytes, s>>>(tm_q, tm_k, tm_v, tm_o, p);
-  return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+  return launch_fwd(tm_q, tm_k, tm_v, tm_o, p, grid, s) == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
 attn_status_t attn_release_host_staging(void) {
@@ -348,6 +377,11 @@ attn_status_t attn_set_option(const char* name, int value) {
   if (std::strcmp(name, "scheduler") == 0) {
     if (value < 0 || value > 2) return ATTN_ERR_UNSUPPORTED;
     g_opt_scheduler.store(value);
+    return ATTN_OK;
+  }
+  if (std::strcmp(name, "kernel") == 0) {
+    if (value < 0 || value > 1) return ATTN_ERR_UNSUPPORTED;
+    g_opt_kernel.store(value);
     return ATTN_OK;
   }
   if (std::strcmp(name, "max_ctas") == 0) {

@@ -67,6 +67,7 @@ struct FwdParams {
   int items_per_group;  // work items per (b, hq) [pair rows] or per (b, hkv) [pair heads]
   int n_work;
   int dynamic;      // 1: work items come from the global counter
+  int kernel;       // which kernel the plan was made for (0: dual query stage, 1: triple score buffer)
   float scale;
   float scale_log2; // scale * log2(e)
   float* lse;

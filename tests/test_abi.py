@@ -69,6 +69,9 @@ def test_options(cdll):
     assert cdll.attn_set_option(None, 1) == 1
     for v in (0, 1, 2):
         assert cdll.attn_set_option(b"scheduler", v) == 0
+    assert cdll.attn_set_option(b"kernel", 2) == 3
+    for v in (1, 0):
+        assert cdll.attn_set_option(b"kernel", v) == 0
     assert cdll.attn_set_option(b"max_ctas", -1) == 3
     assert cdll.attn_set_option(b"max_ctas", 0) == 0
 

@@ -29,9 +29,11 @@ def _library():
     lib.load_library()
     lib.attn_set_option("scheduler", 2)
     lib.attn_set_option("max_ctas", 0)
+    lib.attn_set_option("kernel", 0)
     yield
     lib.attn_set_option("scheduler", 2)
     lib.attn_set_option("max_ctas", 0)
+    lib.attn_set_option("kernel", 0)
 
 
 def run_gpu(q, k, v, causal, scale, want_lse=True, stream=None):
@@ -100,8 +102,16 @@ SMALL = [
 ]
 
 
+@pytest.fixture(params=[0, 1], ids=["dual_stage", "triple_buffer"])
+def kernel(request):
+    """Runs a test once per kernel ("kernel" option of attn_set_option)."""
+    lib.attn_set_option("kernel", request.param)
+    yield request.param
+    lib.attn_set_option("kernel", 0)
+
+
 @pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,causal", SMALL)
-def test_small_cases_match_oracle_everywhere(B, Hq, Hkv, Sq, Sk, causal):
+def test_small_cases_match_oracle_everywhere(kernel, B, Hq, Hkv, Sq, Sk, causal):
     q, k, v = make_qkv(B, Hq, Hkv, Sq, Sk, 128, seed=7000 + Sq + Sk)
     o, lse = run_gpu(q, k, v, causal, SCALE)
     check_full(q, k, v, causal, SCALE, o, lse)
@@ -109,7 +119,7 @@ def test_small_cases_match_oracle_everywhere(B, Hq, Hkv, Sq, Sk, causal):
 
 @pytest.mark.parametrize("sched", [0, 1, 2])
 @pytest.mark.parametrize("max_ctas", [0, 3])
-def test_every_scheduler_mode(sched, max_ctas):
+def test_every_scheduler_mode(kernel, sched, max_ctas):
     lib.attn_set_option("scheduler", sched)
     lib.attn_set_option("max_ctas", max_ctas)
     try:
@@ -123,7 +133,7 @@ def test_every_scheduler_mode(sched, max_ctas):
 
 
 @pytest.mark.parametrize("scale,gain", [(0.5, 1.0), (1e-3, 1.0), (SCALE, 4.0), (SCALE, 8.0)])
-def test_scales_and_peaked_rows(scale, gain):
+def test_scales_and_peaked_rows(kernel, scale, gain):
     """Large score magnitudes move the row maximum by more than the rescale threshold, so the
     accumulator-rescale path runs; tiny scales make softmax nearly uniform."""
     q, k, v = make_qkv(1, 2, 2, 1024, 1024, 128, seed=7200, q_gain=gain)
@@ -133,7 +143,7 @@ def test_scales_and_peaked_rows(scale, gain):
         check_full(q, k, v, causal, scale, o, lse)
 
 
-def test_increasing_scores_force_rescales():
+def test_increasing_scores_force_rescales(kernel):
     """Keys ordered so that every block raises every row's maximum by far more than the
     threshold: each K/V block triggers a rescale of O."""
     B, H, S = 1, 1, 1024
@@ -163,7 +173,7 @@ def test_bitwise_deterministic():
         assert torch.equal(lse.view(torch.int32), outs[0][1].view(torch.int32))
 
 
-def test_zero_q_gives_prefix_means_at_scale():
+def test_zero_q_gives_prefix_means_at_scale(kernel):
     """Q = 0: O is the mean of the visible V rows and LSE = log(#visible keys), a closed form
     that checks masking and block counts of every row at a size the oracle cannot sweep."""
     B, H, S = 1, 4, 8192
@@ -211,6 +221,30 @@ def test_benchmark_workloads_on_sampled_rows(name):
     n_rows = 768 if w.Sk >= 32768 else 1536
     rows = sample_rows(w.B, w.Hq, w.Sq, n_rows, seed=w.seed)
     check_rows(q, k, v, w.causal, w.scale, o, lse, rows)
+
+
+@pytest.mark.parametrize("name", ["mha_causal_s4096", "gqa4_noncausal_s8192", "long_causal_peaked"])
+def test_triple_buffer_kernel_on_benchmark_workloads(name):
+    lib.attn_set_option("kernel", 1)
+    try:
+        test_benchmark_workloads_on_sampled_rows(name)
+    finally:
+        lib.attn_set_option("kernel", 0)
+
+
+def test_decreasing_then_jumping_scores(kernel):
+    """Scores that fall for a while and then jump far above everything seen before: the
+    reference maxima of consecutive K/V blocks differ by hundreds of log2 units."""
+    B, H, S = 1, 1, 1536
+    q = torch.ones((B, S, H, 128), dtype=torch.bfloat16)
+    pos = torch.arange(S, dtype=torch.float32)
+    level = torch.where(pos < 1000, -pos / 8.0, (pos - 900.0) / 4.0).reshape(1, S, 1, 1)
+    k = (level * torch.ones((1, 1, 1, 128))).to(torch.bfloat16)
+    _, _, v = make_qkv(B, H, H, S, S, 128, seed=7350)
+    scale = float(np.float32(1.0 / 16))
+    for causal in (False, True):
+        o, lse = run_gpu(q, k, v, causal, scale)
+        check_full(q, k, v, causal, scale, o, lse)
 
 
 def test_tiny_workload_in_full():

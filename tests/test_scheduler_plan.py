@@ -17,6 +17,9 @@ def _built():
     lib_build.build()
     lib.attn_set_option("scheduler", 2)
     lib.attn_set_option("max_ctas", 0)
+    lib.attn_set_option("kernel", 0)
+    yield
+    lib.attn_set_option("kernel", 0)
 
 
 def visible_blocks_brute(row0, Sq, Sk, causal):
@@ -35,11 +38,16 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("kernel", [0, 1])
 @pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,causal", CASES)
-def test_plan_covers_every_tile_once(B, Hq, Hkv, Sq, Sk, causal):
+def test_plan_covers_every_tile_once(kernel, B, Hq, Hkv, Sq, Sk, causal):
+    lib.attn_set_option("kernel", kernel)
     plan = lib.attn_plan(B, Hq, Hkv, Sq, Sk, 128, causal, 148)
     g = Hq // Hkv
-    assert plan["pair_heads"] == (1 if g % 2 == 0 else 0)
+    if kernel == 1:  # one query tile per work item
+        assert plan["pair_heads"] == 0 and plan["n_work"] == B * Hq * math.ceil(Sq / TILE)
+    else:
+        assert plan["pair_heads"] == (1 if g % 2 == 0 else 0)
     assert plan["n_q_tiles"] == math.ceil(Sq / TILE) and plan["n_kv_blocks"] == math.ceil(Sk / TILE)
     assert plan["ctas"] == min(148, plan["n_work"])
     seen = {}
@@ -64,6 +72,7 @@ def test_plan_covers_every_tile_once(B, Hq, Hkv, Sq, Sk, causal):
 
 
 def test_causal_items_run_longest_first_inside_a_head():
+    lib.attn_set_option("kernel", 0)
     B, H, S = 1, 2, 2048
     plan = lib.attn_plan(B, H, H, S, S, 128, True, 148)
     per = plan["items_per_group"]
@@ -75,6 +84,7 @@ def test_causal_items_run_longest_first_inside_a_head():
 
 
 def test_scheduler_option_changes_grid_only():
+    lib.attn_set_option("kernel", 0)
     lib.attn_set_option("scheduler", 0)
     try:
         plan = lib.attn_plan(2, 16, 16, 16384, 16384, 128, False, 148)
