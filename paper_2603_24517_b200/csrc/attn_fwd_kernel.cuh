@@ -38,7 +38,7 @@ constexpr float kRescaleThreshold = 8.0f;  // log2 units a row maximum may lag b
 #ifndef ATTN_REGS_OTHER
 #define ATTN_REGS_OTHER 64
 #endif
-// Of every four column pairs of a score row, how many take the polynomial exp2 (0..4).
+// Of every eight column pairs of a score row, how many take the polynomial exp2 (0..8).
 #ifndef ATTN_EXP2_POLY_PAIRS
 #define ATTN_EXP2_POLY_PAIRS 1
 #endif
@@ -465,7 +465,7 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
         }
       }
       // P = exp2(S * c - m_used * c) on pairs of columns with packed fp32 arithmetic.  Of every
-      // four pairs, kExp2PolyPairs are evaluated by the polynomial on the FMA pipe and the rest
+      // eight pairs, kExp2PolyPairs are evaluated by the polynomial on the FMA pipe and the rest
       // by the special-function unit, so that neither unit alone bounds the row.
       const float neg_mc = -m_used * c;
       const float2 c2 = make_float2(c, c);
@@ -479,7 +479,7 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
           const int i = cc * 32 + pr * 2;
           const float2 x = fma2(make_float2(X(i), X(i + 1)), c2, nm2);
           float2 e;
-          if ((pr & 3) < kExp2PolyPairs) {
+          if ((pr & 7) < kExp2PolyPairs) {
             e = exp2_poly2(x);
           } else {
             e = make_float2(ex2_approx(x.x), ex2_approx(x.y));

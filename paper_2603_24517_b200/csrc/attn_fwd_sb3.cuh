@@ -331,7 +331,7 @@ __device__ __forceinline__ void role_softmax3(const FwdParams& p, const Bars3& b
             const int i = cc * 32 + pr * 2;
             const float2 x = fma2(make_float2(X(i), X(i + 1)), c2, nm2);
             float2 e;
-            if ((pr & 3) < kExp2PolyPairs) {
+            if ((pr & 7) < kExp2PolyPairs) {
               e = exp2_poly2(x);
             } else {
               e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
@@ -395,7 +395,7 @@ __device__ __forceinline__ void role_softmax3(const FwdParams& p, const Bars3& b
             const int i = cc * 32 + pr * 2;
             const float2 x = fma2(make_float2(X(i), X(i + 1)), c2, nm2);
             float2 e;
-            if ((pr & 3) < kExp2PolyPairs) {
+            if ((pr & 7) < kExp2PolyPairs) {
               e = exp2_poly2(x);
             } else {
               e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
