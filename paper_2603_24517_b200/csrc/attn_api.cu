@@ -148,6 +148,18 @@ void fill_plan(FwdParams* p, int B, int Hq, int Hkv, int Sq, int Sk, int causal)
       p->n_work = B * Hq * p->items_per_group;
     }
   }
+  p->n_groups = p->n_work / p->items_per_group;
+  // Causal: interleave the items of as many heads as keep their K/V (2 tensors x Sk x 128 BF16 per
+  // head) within about 48 MB of L2; non-causal items are all alike, so strict head-major order.
+  p->head_group = 1;
+  if (p->causal) {
+    const long long kv_bytes = 2LL * Sk * attn::kHeadDim * 2;
+    long long g = (48LL << 20) / kv_bytes;
+    if (g < 1) g = 1;
+    if (g > 64) g = 64;
+    if (g > p->n_groups) g = p->n_groups;
+    p->head_group = static_cast<int>(g);
+  }
   p->dynamic = (g_opt_scheduler.load() == 2) ? 1 : 0;
 }
 

@@ -68,6 +68,8 @@ struct FwdParams {
   int n_work;
   int dynamic;      // 1: work items come from the global counter
   int kernel;       // which kernel the plan was made for (0: dual query stage, 1: triple score buffer)
+  int n_groups;     // n_work / items_per_group: (batch, head) groups of work items
+  int head_group;   // groups whose items are interleaved in launch order (1 = strictly group-major)
   float scale;
   float scale_log2; // scale * log2(e)
   float* lse;
@@ -83,9 +85,24 @@ struct Work {
   int nmax;
 };
 
+// Launch order -> (group, rank inside the group).  Groups are (batch, head) units that share K/V;
+// `head_group` consecutive groups are interleaved: rank 0 of each, then rank 1 of each, ...  With
+// the causal mask rank 0 is a group's longest item, so the longest items of several heads start
+// first and the launch ends on short ones, while the K/V of only `head_group` heads is live in L2.
+__host__ __device__ __forceinline__ void split_work(const FwdParams& p, int w, int& grp, int& r) {
+  const int per_super = p.head_group * p.items_per_group;
+  const int sup = w / per_super;
+  const int rem = w - sup * per_super;
+  const int first = sup * p.head_group;
+  int g_eff = p.n_groups - first;
+  if (g_eff > p.head_group) g_eff = p.head_group;
+  r = rem / g_eff;
+  grp = first + (rem - r * g_eff);
+}
+
 __host__ __device__ __forceinline__ void decode_work(const FwdParams& p, int w, Work& wk) {
-  const int grp = w / p.items_per_group;
-  const int r = w - grp * p.items_per_group;
+  int grp, r;
+  split_work(p, w, grp, r);
   if (p.pair_heads) {
     const int hp = p.group >> 1;
     int qt = r / hp;

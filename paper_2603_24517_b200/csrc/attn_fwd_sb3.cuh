@@ -70,10 +70,11 @@ struct Item {
   int b, hq, hkv, row0, n;
 };
 
-// Work item w = one query tile; (batch, head)-major, inside a head longest tiles first when causal.
+// Work item w = one query tile; launch order as in split_work, inside a head longest tiles first
+// when causal.
 __host__ __device__ __forceinline__ void decode_item(const FwdParams& p, int w, Item& it) {
-  const int grp = w / p.n_qt;
-  const int r = w - grp * p.n_qt;
+  int grp, r;
+  split_work(p, w, grp, r);
   const int qt = p.causal ? (p.n_qt - 1 - r) : r;
   it.b = grp / p.Hq;
   it.hq = grp - it.b * p.Hq;

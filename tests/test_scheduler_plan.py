@@ -73,14 +73,31 @@ def test_plan_covers_every_tile_once(kernel, B, Hq, Hkv, Sq, Sk, causal):
 
 def test_causal_items_run_longest_first_inside_a_head():
     lib.attn_set_option("kernel", 0)
-    B, H, S = 1, 2, 2048
+    B, H, S = 2, 3, 2048
     plan = lib.attn_plan(B, H, H, S, S, 128, True, 148)
-    per = plan["items_per_group"]
-    cost = [sum(lib.attn_plan_item(B, H, H, S, S, 128, True, w)[f"n_blocks_{s}"] for s in (0, 1))
-            for w in range(plan["n_work"])]
-    for h in range(B * H):
-        c = cost[h * per:(h + 1) * per]
-        assert c == sorted(c, reverse=True)
+    per_head = {}
+    for w in range(plan["n_work"]):
+        it = lib.attn_plan_item(B, H, H, S, S, 128, True, w)
+        per_head.setdefault((it["b"], it["hq0"]), []).append(it["n_blocks_0"] + it["n_blocks_1"])
+    assert len(per_head) == B * H
+    for costs in per_head.values():
+        assert len(costs) == plan["items_per_group"] and costs == sorted(costs, reverse=True)
+
+
+def test_causal_launch_order_interleaves_heads_and_ends_on_short_items():
+    """Under the causal mask the longest items of several heads go first and the launch ends on
+    the shortest ones (a long item started last would leave the other SMs idle)."""
+    lib.attn_set_option("kernel", 0)
+    B, H, S = 1, 16, 16384
+    plan = lib.attn_plan(B, H, H, S, S, 128, True, 148)
+    first = [lib.attn_plan_item(B, H, H, S, S, 128, True, w) for w in range(6)]
+    assert len({it["hq0"] for it in first}) == 6                       # six different heads ...
+    assert all(it["n_blocks_1"] == plan["n_kv_blocks"] for it in first)  # ... each at its longest item
+    last = lib.attn_plan_item(B, H, H, S, S, 128, True, plan["n_work"] - 1)
+    assert last["n_blocks_0"] + last["n_blocks_1"] == 3
+    # non-causal: strictly head-major
+    nc = [lib.attn_plan_item(B, H, H, S, S, 128, False, w) for w in range(3)]
+    assert {it["hq0"] for it in nc} == {0}
 
 
 def test_scheduler_option_changes_grid_only():
