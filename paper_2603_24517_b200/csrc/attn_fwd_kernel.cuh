@@ -11,8 +11,9 @@
 //   warps 14-15  idle (they only donate registers)
 //
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P aliases the first
-// 64 columns of its S.  Shared memory: Q0, Q1 (32 KB each, reused as the O staging tiles) and a
-// ring of 32 KB K / V tiles, all 128-byte swizzled [128 rows][64 elements] half tiles.
+// 64 columns of its S.  Shared memory: Q0, Q1 (32 KB each), a ring of four 32 KB K / V tiles and one
+// 32 KB O staging tile, all 128-byte swizzled [128 rows][64 elements] half tiles.  The Q tiles of the
+// next work item are fetched as soon as the current item's last Q K^T has been issued.
 #pragma once
 
 #include "ptx.cuh"
@@ -23,7 +24,7 @@ constexpr int kTile = 128;        // rows per Q tile and keys per K/V tile
 constexpr int kHeadDim = 128;
 constexpr int kTileBytes = kTile * kHeadDim * 2;  // 32 KB
 constexpr int kHalfBytes = kTileBytes / 2;        // one [128][64] half tile
-constexpr int kKvSlots = 5;
+constexpr int kKvSlots = 4;
 constexpr int kThreads = 512;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units a row maximum may lag behind
 
@@ -47,11 +48,13 @@ static_assert(8 * ATTN_REGS_SOFTMAX + 4 * ATTN_REGS_EPILOGUE + 4 * ATTN_REGS_OTH
 
 constexpr int kSmemQ = 0;
 constexpr int kSmemKv = 2 * kTileBytes;
-constexpr int kSmemStats = kSmemKv + kKvSlots * kTileBytes;  // float [2 stages][2][128]
+constexpr int kSmemStage = kSmemKv + kKvSlots * kTileBytes;  // O staging tile for the TMA store (both stages, in turn)
+constexpr int kSmemStats = kSmemStage + kTileBytes;          // float [2 stages][2][128]
 constexpr int kSmemBars = kSmemStats + 2 * 2 * kTile * 4;
-constexpr int kNumBars = 2 + 2 + 2 * kKvSlots + 2 * 10;
+constexpr int kNumBars = 2 + 2 + 2 * kKvSlots + 2 * 10 + 1;
 constexpr int kSmemMisc = kSmemBars + kNumBars * 8;  // tmem base, abort flag, sched slots
 constexpr int kSmemBytes = kSmemMisc + 32;
+static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every in-kernel wait gives up after 2 s
 
@@ -174,13 +177,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, WaitCt
 enum : int {
   kRoleLoad = 1 << 8, kRoleMma = 2 << 8, kRoleSoftmax = 3 << 8, kRoleEpilogue = 4 << 8,
   kBarQFull = 1, kBarQEmpty = 2, kBarKvFull = 3, kBarKvEmpty = 4, kBarSFull = 5, kBarPFull = 6,
-  kBarOFull = 7, kBarOEmpty = 8, kBarLFull = 9, kBarLEmpty = 10, kBarSchedFull = 11, kBarSchedEmpty = 12, kBarStFull = 13, kBarPHalf = 14,
+  kBarOFull = 7, kBarOEmpty = 8, kBarLFull = 9, kBarLEmpty = 10, kBarSchedFull = 11, kBarSchedEmpty = 12, kBarStFull = 13, kBarPHalf = 14, kBarStgEmpty = 18,
   kBadSmemAlign = 0x7001
 };
 
 struct Barriers {
   uint64_t* q_full;    // [2]  loader (TMA tx) -> MMA
-  uint64_t* q_empty;   // [2]  epilogue (TMA store has read the staging tile) -> loader
+  uint64_t* q_empty;   // [2]  MMA commit after the item's last Q K^T of that stage -> loader
   uint64_t* kv_full;   // [kKvSlots]
   uint64_t* kv_empty;  // [kKvSlots]  MMA commit -> loader
   uint64_t* s_full;    // [2]  MMA commit -> softmax
@@ -191,6 +194,7 @@ struct Barriers {
   uint64_t* l_full;    // [2]  softmax (128 threads) -> epilogue
   uint64_t* l_empty;   // [2]  epilogue (128 threads) -> softmax
   uint64_t* st_full;   // [2]  epilogue (4 warps: staging tile written) -> the thread issuing the TMA store
+  uint64_t* stg_empty; // [1]  the thread that issued the TMA store (source read) -> epilogue warps
   uint64_t* sched_full;   // [2]  loader -> every consumer role
   uint64_t* sched_empty;  // [2]  13 consumer arrivals -> loader
 };
@@ -345,7 +349,10 @@ __device__ __forceinline__ void role_mma(const FwdParams& p, const Barriers& bar
           if (!mbar_wait_warp(&bars.q_full[s], q_cnt[s] & 1, ctx, kRoleMma | kBarQFull)) return;
           tc_fence_after_sync();
           issue_qk(leader, tmem + s * kTile, q_desc[s], k_desc);
-          if (leader) mma_commit(&bars.s_full[s]);
+          if (leader) {
+            mma_commit(&bars.s_full[s]);
+            if (wk.n[s] == 1) mma_commit(&bars.q_empty[s]);  // Q_s is not read again
+          }
         }
       }
       if (leader) mma_commit(&bars.kv_empty[slot]);
@@ -388,7 +395,10 @@ __device__ __forceinline__ void role_mma(const FwdParams& p, const Barriers& bar
               k_ready = true;
             }
             issue_qk(leader, tmem + s * kTile, q_desc[s], k_desc);
-            if (leader) mma_commit(&bars.s_full[s]);
+            if (leader) {
+              mma_commit(&bars.s_full[s]);
+              if (j + 2 == wk.n[s]) mma_commit(&bars.q_empty[s]);  // that was the item's last use of Q_s
+            }
           }
         }
       }
@@ -538,6 +548,7 @@ __device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers
                                               int row_in_tile, int lane, const CUtensorMap* tm_o) {
   const uint32_t lane_sel = static_cast<uint32_t>(row_in_tile & ~31) << 16;
   uint32_t cnt[2] = {0, 0};
+  uint32_t stg_cnt = 0;  // uses of the staging tile so far (phase of stg_empty)
   for (int it = 0;; ++it) {
     const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleEpilogue, lane == 0, true);
     if (w < 0 || w >= p.n_work) return;
@@ -559,7 +570,12 @@ __device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers
       ++cnt[s];
       tc_fence_after_sync();
       const float inv_l = 1.0f / l;
-      uint8_t* stage = smem + kSmemQ + s * kTileBytes;  // the Q_s tile is dead once o_full[s] fired
+      // the previous TMA store must have finished reading the staging tile
+      ok = mbar_wait(&bars.stg_empty[0], (stg_cnt & 1) ^ 1, ctx, kRoleEpilogue | kBarStgEmpty);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return;
+      ++stg_cnt;
+      uint8_t* stage = smem + kSmemStage;
       const uint32_t t_o = tmem + lane_sel + 2 * kTile + s * kTile;
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
@@ -595,7 +611,7 @@ __device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers
           tma_store_4d(tm_o, stage + kHalfBytes, 64, wk.hq[s], wk.row0[s], wk.b);
           tma_store_commit();
           tma_store_wait_read0();
-          mbar_arrive(&bars.q_empty[s]);
+          mbar_arrive(&bars.stg_empty[0]);
         }
       }
     }
@@ -625,7 +641,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   bars.l_full = bars.o_empty + 2;
   bars.l_empty = bars.l_full + 2;
   bars.st_full = bars.l_empty + 2;
-  bars.sched_full = bars.st_full + 2;
+  bars.stg_empty = bars.st_full + 2;
+  bars.sched_full = bars.stg_empty + 1;
   bars.sched_empty = bars.sched_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kSmemMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kSmemMisc + 4);
@@ -652,6 +669,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(&bars.l_full[i], kTile);
       mbar_init(&bars.l_empty[i], kTile);
       mbar_init(&bars.st_full[i], 4);
+      if (i == 0) mbar_init(&bars.stg_empty[0], 1);
       mbar_init(&bars.sched_full[i], 1);
       mbar_init(&bars.sched_empty[i], kSchedConsumers);
     }
