@@ -150,15 +150,27 @@ void fill_plan(FwdParams* p, int B, int Hq, int Hkv, int Sq, int Sk, int causal)
   }
   p->n_groups = p->n_work / p->items_per_group;
   // Causal: interleave the items of as many heads as keep their K/V (2 tensors x Sk x 128 BF16 per
-  // head) within about 48 MB of L2; non-causal items are all alike, so strict head-major order.
+  // head) within about 72 MB of L2 (measured best of 24..100 MB); non-causal items are all alike, so strict head-major order.
   p->head_group = 1;
+  p->head_group_extra = p->n_groups;  // every super-group is one group
   if (p->causal) {
     const long long kv_bytes = 2LL * Sk * attn::kHeadDim * 2;
-    long long g = (48LL << 20) / kv_bytes;
+    long long g = (72LL << 20) / kv_bytes;
     if (g < 1) g = 1;
     if (g > 64) g = 64;
     if (g > p->n_groups) g = p->n_groups;
-    p->head_group = static_cast<int>(g);
+    // k super-groups of nearly equal size (they differ by at most one group), so that the last
+    // one is not a small remainder whose long items would start when little other work is left
+    const int k = static_cast<int>((p->n_groups + g - 1) / g);
+    const int base = p->n_groups / k;
+    const int extra = p->n_groups % k;
+    if (extra == 0) {
+      p->head_group = base;
+      p->head_group_extra = k;
+    } else {
+      p->head_group = base + 1;
+      p->head_group_extra = extra;
+    }
   }
   p->dynamic = (g_opt_scheduler.load() == 2) ? 1 : 0;
 }

@@ -72,7 +72,8 @@ struct FwdParams {
   int dynamic;      // 1: work items come from the global counter
   int kernel;       // which kernel the plan was made for (0: dual query stage, 1: triple score buffer)
   int n_groups;     // n_work / items_per_group: (batch, head) groups of work items
-  int head_group;   // groups whose items are interleaved in launch order (1 = strictly group-major)
+  int head_group;   // groups per large super-group (1 = strictly group-major launch order)
+  int head_group_extra;  // how many super-groups are large; the others hold head_group - 1 groups
   float scale;
   float scale_log2; // scale * log2(e)
   float* lse;
@@ -88,17 +89,28 @@ struct Work {
   int nmax;
 };
 
-// Launch order -> (group, rank inside the group).  Groups are (batch, head) units that share K/V;
-// `head_group` consecutive groups are interleaved: rank 0 of each, then rank 1 of each, ...  With
-// the causal mask rank 0 is a group's longest item, so the longest items of several heads start
-// first and the launch ends on short ones, while the K/V of only `head_group` heads is live in L2.
+// Launch order -> (group, rank inside the group).  Groups are (batch, head) units that share K/V.
+// Consecutive groups form super-groups of `head_group` (the first `head_group_extra` of them) or
+// `head_group - 1` groups, whose items are interleaved: rank 0 of each group, then rank 1 of each,
+// ...  With the causal mask rank 0 is a group's longest item, so the longest items of several
+// heads start first and every super-group -- the last one too -- ends on short ones, while only a
+// super-group's K/V is live in L2.
 __host__ __device__ __forceinline__ void split_work(const FwdParams& p, int w, int& grp, int& r) {
-  const int per_super = p.head_group * p.items_per_group;
-  const int sup = w / per_super;
-  const int rem = w - sup * per_super;
-  const int first = sup * p.head_group;
-  int g_eff = p.n_groups - first;
-  if (g_eff > p.head_group) g_eff = p.head_group;
+  const int big = p.head_group * p.items_per_group;  // items of a large super-group
+  const int n_big_items = p.head_group_extra * big;
+  int first, g_eff, rem;
+  if (w < n_big_items) {
+    const int sup = w / big;
+    rem = w - sup * big;
+    first = sup * p.head_group;
+    g_eff = p.head_group;
+  } else {
+    const int small = big - p.items_per_group;  // head_group - 1 groups (never empty here)
+    const int sup = (w - n_big_items) / small;
+    rem = (w - n_big_items) - sup * small;
+    first = p.head_group_extra * p.head_group + sup * (p.head_group - 1);
+    g_eff = p.head_group - 1;
+  }
   r = rem / g_eff;
   grp = first + (rem - r * g_eff);
 }
