@@ -165,6 +165,17 @@ int attn_version(void);
  */
 attn_status_t attn_last_device_status(int* code, int* detail);
 
+/*
+ * attn_selftest_wait_timeout -- exercises the bounded waits every kernel of this library uses
+ * between its warp roles (the paper's kernels hand work between MMA, softmax, correction and
+ * load warps "with barrier-based signaling", Section 2.2; here every such wait has a time limit).
+ * Launches one warp that waits on a barrier nobody signals; after `limit_ms` (1..1000) the wait
+ * gives up, the kernel returns normally and attn_last_device_status() reports ATTN_ERR_TIMEOUT
+ * with *code = 0x905.  Nothing faults or hangs; later calls on the device work as usual.
+ * Asynchronous on `stream`.
+ */
+attn_status_t attn_selftest_wait_timeout(int limit_ms, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,7 @@ STATUS_NAMES = {
     5: "ATTN_ERR_CUDA", 6: "ATTN_ERR_ARCH", 7: "ATTN_ERR_TIMEOUT", 8: "ATTN_ERR_TOO_LARGE",
 }
 EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_host", "attn_fwd_noalloc", "attn_release_host_staging", "attn_set_option",
-                    "attn_plan", "attn_plan_item", "attn_status_str", "attn_version",
+                    "attn_plan", "attn_plan_item", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
                     "attn_last_device_status")
 
 _lib = None
@@ -58,6 +58,8 @@ def load_library() -> ctypes.CDLL:
     lib.attn_plan.restype = ci
     lib.attn_plan_item.argtypes = [ci] * 8 + [ctypes.POINTER(ci)]
     lib.attn_plan_item.restype = ci
+    lib.attn_selftest_wait_timeout.argtypes = [ci, vp]
+    lib.attn_selftest_wait_timeout.restype = ci
     lib.attn_status_str.argtypes = [ci]
     lib.attn_status_str.restype = ctypes.c_char_p
     lib.attn_version.argtypes = []
@@ -168,6 +170,18 @@ def attn_plan_item(B, Hq, Hkv, Sq, Sk, D, causal, w) -> dict:
         raise AttnError(st, "attn_plan_item")
     keys = ("b", "hkv", "hq0", "hq1", "row0_0", "row0_1", "n_blocks_0", "n_blocks_1")
     return dict(zip(keys, list(out)))
+
+
+def attn_selftest_wait_timeout(limit_ms: int, device=0, stream=None) -> None:
+    """Launches the bounded-wait self-test (see include/attn.h); read the outcome with
+    ``attn_last_device_status``."""
+    dev = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
+    if stream is None:
+        stream = torch.cuda.current_stream(dev).cuda_stream
+    with torch.cuda.device(dev):
+        st = load_library().attn_selftest_wait_timeout(int(limit_ms), stream)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_selftest_wait_timeout")
 
 
 def attn_status_str(status: int) -> str:

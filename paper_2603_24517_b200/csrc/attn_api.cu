@@ -416,6 +416,16 @@ attn_status_t attn_set_option(const char* name, int value) {
   return ATTN_ERR_UNSUPPORTED;
 }
 
+attn_status_t attn_selftest_wait_timeout(int limit_ms, void* stream) {
+  if (limit_ms < 1 || limit_ms > 1000) return ATTN_ERR_UNSUPPORTED;
+  attn_status_t st = ATTN_OK;
+  DeviceState* dev = device_state(&st);
+  if (dev == nullptr) return st;
+  attn::wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      dev->status, static_cast<uint64_t>(limit_ms) * 1000000ull);
+  return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
 const char* attn_status_str(attn_status_t status) {
   switch (status) {
     case ATTN_OK: return "ATTN_OK";

@@ -152,12 +152,13 @@ __host__ __device__ __forceinline__ void decode_work(const FwdParams& p, int w, 
 }
 
 // ------------------------------------------------------------------------------------------
-// Bounded mbarrier wait.  Returns false after kWaitLimitNs, or as soon as any thread of the
+// Bounded mbarrier wait.  Returns false after ctx.limit_ns, or as soon as any thread of the
 // CTA has given up; the first to give up records (code, detail) in the global status word.
 // ------------------------------------------------------------------------------------------
 struct WaitCtx {
   volatile int* abort_flag;  // shared memory
   int* status;               // global
+  uint64_t limit_ns;         // how long one wait may last
 };
 
 __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, WaitCtx ctx, int code) {
@@ -173,7 +174,7 @@ __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, W
     if (*ctx.abort_flag) return false;
     const uint64_t now = global_timer_ns();
     if (t0 == 0) t0 = now;
-    if (now - t0 > kWaitLimitNs) {
+    if (now - t0 > ctx.limit_ns) {
       *ctx.abort_flag = 1;
       if (atomicCAS(ctx.status, 0, code) == 0) ctx.status[1] = static_cast<int>(blockIdx.x);
       return false;
@@ -190,7 +191,8 @@ enum : int {
   kRoleLoad = 1 << 8, kRoleMma = 2 << 8, kRoleSoftmax = 3 << 8, kRoleEpilogue = 4 << 8,
   kBarQFull = 1, kBarQEmpty = 2, kBarKvFull = 3, kBarKvEmpty = 4, kBarSFull = 5, kBarPFull = 6,
   kBarOFull = 7, kBarOEmpty = 8, kBarLFull = 9, kBarLEmpty = 10, kBarSchedFull = 11, kBarSchedEmpty = 12, kBarStFull = 13, kBarPHalf = 14, kBarStgEmpty = 18,
-  kBadSmemAlign = 0x7001
+  kBadSmemAlign = 0x7001,
+  kRoleSelfTest = 9 << 8
 };
 
 struct Barriers {
@@ -659,7 +661,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kSmemMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kSmemMisc + 4);
   volatile int* sched_w = reinterpret_cast<volatile int*>(smem + kSmemMisc + 8);
-  const WaitCtx ctx{abort_flag, p.status};
+  const WaitCtx ctx{abort_flag, p.status, kWaitLimitNs};
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -735,6 +737,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tc_fence_after_sync();
     tmem_dealloc(tmem, 512);
   }
+}
+
+// Self-test of the bounded wait: one warp waits on an mbarrier that nobody ever arrives on.  The
+// wait gives up after limit_ns, records (kRoleSelfTest | kBarSFull, block) in the status word and
+// the kernel returns normally, leaving the context usable.
+__global__ void __launch_bounds__(32, 1) wait_timeout_selftest_kernel(int* status, uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  __syncwarp();
+  const WaitCtx ctx{&abort_flag, status, limit_ns};
+  mbar_wait_warp(&bar, 0, ctx, kRoleSelfTest | kBarSFull);
 }
 
 }  // namespace attn

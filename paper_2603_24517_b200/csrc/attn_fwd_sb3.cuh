@@ -524,7 +524,7 @@ attn_fwd_sb3_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kSmemMisc3);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kSmemMisc3 + 4);
   volatile int* sched_w = reinterpret_cast<volatile int*>(smem + kSmemMisc3 + 8);
-  const WaitCtx ctx{abort_flag, p.status};
+  const WaitCtx ctx{abort_flag, p.status, kWaitLimitNs};
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;

@@ -78,6 +78,8 @@ def test_options(cdll):
 
 def test_last_device_status_null(cdll):
     assert cdll.attn_last_device_status(None, None) == 1
+    assert cdll.attn_selftest_wait_timeout(0, None) == 3
+    assert cdll.attn_selftest_wait_timeout(5000, None) == 3
 
 
 def test_missing_library_is_loud(monkeypatch):

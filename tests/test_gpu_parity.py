@@ -200,6 +200,22 @@ def test_host_entry_point_matches_device_entry_point():
     lib.attn_release_host_staging()
 
 
+def test_expired_wait_is_reported_and_the_device_stays_usable():
+    """A wait that nothing satisfies runs into its time limit: the kernel returns, the status
+    word names the waiter, and the next launches work."""
+    import time
+    t0 = time.perf_counter()
+    lib.attn_selftest_wait_timeout(20)
+    st, code, detail = lib.attn_last_device_status()
+    assert time.perf_counter() - t0 < 5.0
+    assert st == 7 and lib.attn_status_str(st) == "ATTN_ERR_TIMEOUT"
+    assert code == 0x905 and detail == 0
+    assert lib.attn_last_device_status() == (0, 0, 0)  # reading clears it
+    q, k, v = make_qkv(1, 2, 2, 256, 256, 128, seed=7900)
+    o, lse = run_gpu(q, k, v, True, SCALE)
+    check_full(q, k, v, True, SCALE, o, lse)
+
+
 def test_error_statuses_on_device_tensors():
     q, k, v = (t.cuda() for t in make_qkv(1, 2, 2, 256, 128, 128, seed=7800))
     o = torch.empty_like(q)
