@@ -122,6 +122,15 @@ attn_status_t attn_release_host_staging(void);
  *                 1 = persistent CTAs, static round-robin over work items
  *                 2 = persistent CTAs, dynamic work counter (default)
  *   "max_ctas"    0 = one per SM (default), else an upper bound on persistent CTAs
+ *   "rescale_threshold"  0..64 (default 8): log2 units by which a row's reference maximum may
+ *                 lag its true running maximum before the O accumulator is rescaled; 0 rescales
+ *                 whenever the maximum moves (the paper's Section 5.1 discusses this step)
+ *   "split_p"     1 (default) = P is handed to the MMA warp in two halves of 64 keys, so the
+ *                 first half of P V overlaps the second half of the exponentials; 0 = in one piece
+ *                 ("kernel" = 0 only)
+ *   "overlap_epilogue"  1 (default) = a query stage is normalised and stored as soon as its own
+ *                 last P V has completed, overlapping the other stage's (Section 5.2);
+ *                 0 = only after both stages' last P V ("kernel" = 0 only)
  *   "kernel"      0 = dual query stage: a CTA runs two 128-row query tiles against one stream
  *                     of K/V tiles, one score buffer each (default)
  *                 1 = triple score buffer: a CTA runs one query tile with three score tiles

@@ -38,6 +38,9 @@ EncodeTiledFn g_encode = nullptr;
 std::atomic<int> g_opt_scheduler{2};
 std::atomic<int> g_opt_max_ctas{0};
 std::atomic<int> g_opt_kernel{0};  // 0: dual query stage, 1: triple score buffer
+std::atomic<int> g_opt_rescale_threshold{8};
+std::atomic<int> g_opt_split_p{1};
+std::atomic<int> g_opt_overlap_epilogue{1};
 
 // Per-device one-time set-up: architecture check, kernel attribute, scheduler counters and
 // status word.  Returns the state or nullptr (with *st set).
@@ -173,6 +176,9 @@ void fill_plan(FwdParams* p, int B, int Hq, int Hkv, int Sq, int Sk, int causal)
     }
   }
   p->dynamic = (g_opt_scheduler.load() == 2) ? 1 : 0;
+  p->rescale_threshold = static_cast<float>(g_opt_rescale_threshold.load());
+  p->split_p = g_opt_split_p.load();
+  p->overlap_epilogue = g_opt_overlap_epilogue.load();
 }
 
 // Launches the kernel selected by the "kernel" option (the plan in `p` was made for it).
@@ -406,6 +412,21 @@ attn_status_t attn_set_option(const char* name, int value) {
   if (std::strcmp(name, "kernel") == 0) {
     if (value < 0 || value > 1) return ATTN_ERR_UNSUPPORTED;
     g_opt_kernel.store(value);
+    return ATTN_OK;
+  }
+  if (std::strcmp(name, "rescale_threshold") == 0) {
+    if (value < 0 || value > 64) return ATTN_ERR_UNSUPPORTED;
+    g_opt_rescale_threshold.store(value);
+    return ATTN_OK;
+  }
+  if (std::strcmp(name, "split_p") == 0) {
+    if (value < 0 || value > 1) return ATTN_ERR_UNSUPPORTED;
+    g_opt_split_p.store(value);
+    return ATTN_OK;
+  }
+  if (std::strcmp(name, "overlap_epilogue") == 0) {
+    if (value < 0 || value > 1) return ATTN_ERR_UNSUPPORTED;
+    g_opt_overlap_epilogue.store(value);
     return ATTN_OK;
   }
   if (std::strcmp(name, "max_ctas") == 0) {

@@ -26,7 +26,7 @@ constexpr int kTileBytes = kTile * kHeadDim * 2;  // 32 KB
 constexpr int kHalfBytes = kTileBytes / 2;        // one [128][64] half tile
 constexpr int kKvSlots = 4;
 constexpr int kThreads = 512;
-constexpr float kRescaleThreshold = 8.0f;  // log2 units a row maximum may lag behind
+constexpr float kRescaleThreshold = 8.0f;  // default log2 units a row maximum may lag behind
 
 // Registers per thread of each role after the setmaxnreg re-split of the CTA's 64K registers:
 // 8 softmax warps, 4 epilogue warps, 4 other warps; 8 * a + 4 * b + 4 * c must not exceed 2048.
@@ -74,6 +74,9 @@ struct FwdParams {
   int n_groups;     // n_work / items_per_group: (batch, head) groups of work items
   int head_group;   // groups per large super-group (1 = strictly group-major launch order)
   int head_group_extra;  // how many super-groups are large; the others hold head_group - 1 groups
+  float rescale_threshold;  // log2 units a row's reference maximum may lag before O is rescaled
+  int split_p;              // 1: P is released to the MMA warp in two halves of 64 keys
+  int overlap_epilogue;     // 1: a stage is normalised and stored as soon as its own last P V is done
   float scale;
   float scale_log2; // scale * log2(e)
   float* lse;
@@ -488,7 +491,7 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
         m_used = (m_blk == -INFINITY) ? 0.f : m_blk;
       } else {
         const float m_new = fmaxf(m_used, m_blk);
-        const bool grow = (m_new - m_used) * c > kRescaleThreshold;
+        const bool grow = (m_new - m_used) * c > p.rescale_threshold;
         if (__any_sync(0xffffffffu, grow)) {
           // P V of block j-1 has completed (S of block j was issued after it), so O_s is quiescent
           const float alpha = ex2_approx((m_used - m_new) * c);
@@ -533,7 +536,7 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
           pk[pr] = pack_bf16x2(e.x, e.y);
         }
         tmem_st_x16(t_s + cc * 16, pk);
-        if (cc == 1) {  // the first 64 keys of P are in tensor memory
+        if (cc == 1 && p.split_p) {  // the first 64 keys of P are in tensor memory
           tmem_wait_st();
           tc_fence_before_sync();
           if (lane == 0) mbar_arrive(&bars.p_half[s]);
@@ -544,7 +547,10 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
       l += la.x + la.y;
       tmem_wait_st();
       tc_fence_before_sync();
-      if (lane == 0) mbar_arrive(&bars.p_full[s]);
+      if (lane == 0) {
+        if (!p.split_p) mbar_arrive(&bars.p_half[s]);
+        mbar_arrive(&bars.p_full[s]);
+      }
     }
     // hand the row statistics to the epilogue warps
     bool ok = mbar_wait(&bars.l_empty[s], (l_cnt & 1) ^ 1, ctx, kRoleSoftmax | kBarLEmpty);
@@ -581,6 +587,12 @@ __device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers
       ok = mbar_wait(&bars.o_full[s], cnt[s] & 1, ctx, kRoleEpilogue | kBarOFull);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) return;
+      if (!p.overlap_epilogue && s == 0 && wk.n[1] > 0) {
+        // A/B switch: do not start on stage 0 before stage 1's last P V has completed as well
+        ok = mbar_wait(&bars.o_full[1], cnt[1] & 1, ctx, kRoleEpilogue | kBarOFull);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) return;
+      }
       ++cnt[s];
       tc_fence_after_sync();
       const float inv_l = 1.0f / l;

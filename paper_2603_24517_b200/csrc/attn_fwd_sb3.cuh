@@ -308,7 +308,7 @@ __device__ __forceinline__ void role_softmax3(const FwdParams& p, const Bars3& b
       if (cand == -INFINITY) {
         m_cur = (own_max == -INFINITY) ? 0.f : own_max;
       } else {
-        m_cur = ((own_max - cand) * c > kRescaleThreshold) ? own_max : cand;
+        m_cur = ((own_max - cand) * c > p.rescale_threshold) ? own_max : cand;
       }
       const int my_slot = ((g * 2) + ((j >> 1) & 1)) * kTile + row_in_tile;
       float2 la, lb;

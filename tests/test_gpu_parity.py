@@ -132,6 +132,24 @@ def test_every_scheduler_mode(kernel, sched, max_ctas):
         lib.attn_set_option("max_ctas", 0)
 
 
+@pytest.mark.parametrize("option,value", [("rescale_threshold", 0), ("rescale_threshold", 2), ("rescale_threshold", 64),
+                                          ("split_p", 0), ("overlap_epilogue", 0)])
+def test_design_switches_keep_the_result(kernel, option, value):
+    lib.attn_set_option(option, value)
+    try:
+        # a reference that may lag by 2^64 leaves the dominant weights of peaked rows inexact in BF16,
+        # which adds up to ~8e-3 to |dO| there: peaked inputs only with the tighter settings
+        gains = (1.0, 1.0) if (option, value) == ("rescale_threshold", 64) else (4.0, 1.0)
+        for (B, Hq, Hkv, Sq, Sk, causal), gain in zip([(1, 4, 4, 900, 900, True), (2, 4, 2, 384, 1000, False)], gains):
+            q, k, v = make_qkv(B, Hq, Hkv, Sq, Sk, 128, seed=7150, q_gain=gain)
+            o, lse = run_gpu(q, k, v, causal, SCALE)
+            check_full(q, k, v, causal, SCALE, o, lse)
+    finally:
+        lib.attn_set_option("rescale_threshold", 8)
+        lib.attn_set_option("split_p", 1)
+        lib.attn_set_option("overlap_epilogue", 1)
+
+
 @pytest.mark.parametrize("scale,gain", [(0.5, 1.0), (1e-3, 1.0), (SCALE, 4.0), (SCALE, 8.0)])
 def test_scales_and_peaked_rows(kernel, scale, gain):
     """Large score magnitudes move the row maximum by more than the rescale threshold, so the
