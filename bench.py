@@ -50,6 +50,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--op", default="fwd", choices=["fwd", "merge"],
+                    help="fwd: the attention forward (default, the headline metric); merge: the LSE-weighted "
+                         "merge of two partial results of the same shape (HBM-bound side kernel)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target oracle time of the cpu_baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -302,6 +305,54 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_merge(args, w):
+    """attn_merge on two partial results shaped like the workload's O / LSE: GB/s against the
+    measured HBM copy bandwidth.  One GPU."""
+    import paper_2603_24517_b200 as lib
+    from paper_2603_24517_b200 import build as lib_build
+    lib_build.build()
+    lib.load_library()
+    dev = torch.device("cuda", 0)
+    g = torch.Generator(device=dev)
+    g.manual_seed(w.seed)
+    shape = (w.B, w.Sq, w.Hq, w.D)
+    o1 = torch.randn(shape, device=dev, generator=g).to(torch.bfloat16)
+    o2 = torch.randn(shape, device=dev, generator=g).to(torch.bfloat16)
+    l1 = torch.randn((w.B, w.Hq, w.Sq), device=dev, generator=g)
+    l2 = torch.randn((w.B, w.Hq, w.Sq), device=dev, generator=g)
+    o = torch.empty_like(o1)
+    lse = torch.empty_like(l1)
+    rows = w.B * w.Sq * w.Hq
+    algorithmic = rows * (3 * w.D * 2 + 3 * 4)  # read O1, O2, LSE1, LSE2; write O, LSE
+    for _ in range(max(3, args.warmup)):
+        lib.attn_merge(o1, l1, o2, l2, o, lse)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        lib.attn_merge(o1, l1, o2, l2, o, lse)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    gbs = algorithmic / (ms * 1e-3) / 1e9
+    peak = 6650.0
+    kind = "fallback"
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            peak = float(json.load(f)["hbm_gbs"])
+        kind = "measured"
+    print(json.dumps({
+        "metric": "attn_merge_gbs", "value": gbs, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "dtype": "f32",
+        "data": "synthetic", "gpu_launches": args.steps,
+        "config": {"workload": f"merge of two partial results shaped like {w.name}", "rows": rows,
+                   "l2": f"{algorithmic / 2**20:.0f} MiB per launch exceed the 126 MB L2; no flush"},
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                     "peak_kind": f"{kind} copy bandwidth", "traffic": None, "algorithmic_bytes": algorithmic},
+    }), flush=True)
+
+
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
 # profiles/ (None until a capture of the current kernel exists).
 TRAFFIC_BYTES: dict[str, float | None] = {}
@@ -313,7 +364,9 @@ def main():
     if args.workload not in workloads:
         raise SystemExit(f"unknown workload {args.workload}; choose from {sorted(workloads)}")
     w = workloads[args.workload]
-    if args.impl == "reference":
+    if args.op == "merge":
+        run_merge(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)

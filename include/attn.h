@@ -175,6 +175,27 @@ int attn_version(void);
 attn_status_t attn_last_device_status(int* code, int* detail);
 
 /*
+ * attn_merge -- combines two partial attention results that were computed over DISJOINT sets of
+ * keys for the same queries (e.g. two attn_fwd calls on the two halves of K and V, non-causal):
+ *
+ *     LSE = log(exp(LSE1) + exp(LSE2)),   O = exp(LSE1 - LSE) * O1 + exp(LSE2 - LSE) * O2
+ *
+ * which is the attention over the union of the keys -- a direct consequence of the softmax
+ * definition of Section 2.2 and the reason attn_fwd returns LSE.  It is what a caller needs to
+ * split a long key sequence over several launches or devices.
+ *
+ *   o1, o2   BF16 [B, Sq, Hq, D] device pointers (read), 16-byte aligned
+ *   lse1/2   FP32 [B, Hq, Sq] (read); -inf marks a part that saw no key (weight 0)
+ *   o        BF16 [B, Sq, Hq, D] (written; may be the same buffer as o1 or o2)
+ *   lse      FP32 [B, Hq, Sq]    (written; must not alias lse1 or lse2)
+ *   D        must be 128
+ * Asynchronous on `stream`.  Arithmetic in fp32, O rounded to nearest-even BF16.  If both parts
+ * are empty the row is O = 0, LSE = -inf.
+ */
+attn_status_t attn_merge(const void* o1, const float* lse1, const void* o2, const float* lse2,
+                         void* o, float* lse, int B, int Hq, int Sq, int D, void* stream);
+
+/*
  * attn_selftest_wait_timeout -- exercises the bounded waits every kernel of this library uses
  * between its warp roles (the paper's kernels hand work between MMA, softmax, correction and
  * load warps "with barrier-based signaling", Section 2.2; here every such wait has a time limit).

@@ -191,3 +191,32 @@ int attn_oracle_weights(const uint16_t *q, const uint16_t *k, const uint16_t *v,
     free(o_row);
     return 0;
 }
+
+/*
+ * Merge of two partial attention results over disjoint key sets (the identity behind
+ * splitting the key sequence, a direct consequence of the softmax definition in Section 2.2):
+ * with LSE = log(exp(LSE1) + exp(LSE2)) and w_i = exp(LSE_i - LSE),  O = w1 O1 + w2 O2.
+ * o1, o2: BF16 bit patterns [rows, D]; lse1, lse2: fp32 [rows] (as the GPU library stores them);
+ * o: double [rows, D]; lse: double [rows].  A part with LSE = -inf (no visible key) has weight 0;
+ * if both parts are empty the row is O = 0, LSE = -inf.
+ */
+int attn_oracle_merge(const uint16_t *o1, const float *lse1, const uint16_t *o2, const float *lse2,
+                      int64_t rows, int64_t D, double *o, double *lse)
+{
+    if (rows <= 0 || D <= 0) return 1;
+    for (int64_t r = 0; r < rows; ++r) {
+        const double a = (double)lse1[r], b = (double)lse2[r];
+        const double m = a > b ? a : b;
+        if (m == -INFINITY) {
+            lse[r] = -INFINITY;
+            for (int64_t d = 0; d < D; ++d) o[r * D + d] = 0.0;
+            continue;
+        }
+        const double tot = m + log(exp(a - m) + exp(b - m));
+        const double w1 = exp(a - tot), w2 = exp(b - tot);
+        lse[r] = tot;
+        for (int64_t d = 0; d < D; ++d)
+            o[r * D + d] = w1 * bf16_to_double(o1[r * D + d]) + w2 * bf16_to_double(o2[r * D + d]);
+    }
+    return 0;
+}

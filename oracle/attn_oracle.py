@@ -55,6 +55,9 @@ def _load():
             lib.attn_oracle_weights.argtypes = [u16p, u16p, u16p, *shape, ctypes.c_int, ctypes.c_float,
                                                 i64, i64, i64, f64p]
             lib.attn_oracle_weights.restype = ctypes.c_int
+            f32p = ctypes.POINTER(ctypes.c_float)
+            lib.attn_oracle_merge.argtypes = [u16p, f32p, u16p, f32p, i64, i64, f64p, f64p]
+            lib.attn_oracle_merge.restype = ctypes.c_int
             _lib = lib
     return _lib
 
@@ -122,3 +125,25 @@ def softmax_weights(q, k, v, causal: bool, scale: float, b: int, hq: int, i: int
     if rc != 0:
         raise ValueError(f"attn_oracle_weights failed with code {rc}")
     return p
+
+
+def merge(o1, lse1, o2, lse2):
+    """LSE-weighted merge of two partial results over disjoint key sets.
+    o1, o2: uint16 BF16 bits [..., D]; lse1, lse2: float32 [...] with one entry per row of o
+    (same row order).  Returns (O float64 [..., D], LSE float64 [...])."""
+    o1 = np.ascontiguousarray(o1, dtype=np.uint16)
+    o2 = np.ascontiguousarray(o2, dtype=np.uint16)
+    lse1 = np.ascontiguousarray(lse1, dtype=np.float32)
+    lse2 = np.ascontiguousarray(lse2, dtype=np.float32)
+    D = o1.shape[-1]
+    rows = o1.size // D
+    if o2.shape != o1.shape or lse1.size != rows or lse2.size != rows:
+        raise ValueError("inconsistent shapes")
+    o = np.empty(o1.shape, dtype=np.float64)
+    lse = np.empty(lse1.shape, dtype=np.float64)
+    rc = _load().attn_oracle_merge(_p(o1, ctypes.c_uint16), _p(lse1, ctypes.c_float), _p(o2, ctypes.c_uint16),
+                                   _p(lse2, ctypes.c_float), rows, D, _p(o, ctypes.c_double),
+                                   _p(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"attn_oracle_merge failed with code {rc}")
+    return o, lse

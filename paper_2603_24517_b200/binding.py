@@ -20,7 +20,7 @@ STATUS_NAMES = {
     0: "ATTN_OK", 1: "ATTN_ERR_NULL", 2: "ATTN_ERR_SHAPE", 3: "ATTN_ERR_UNSUPPORTED", 4: "ATTN_ERR_ALIGN",
     5: "ATTN_ERR_CUDA", 6: "ATTN_ERR_ARCH", 7: "ATTN_ERR_TIMEOUT", 8: "ATTN_ERR_TOO_LARGE",
 }
-EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_host", "attn_fwd_noalloc", "attn_release_host_staging", "attn_set_option",
+EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_host", "attn_fwd_noalloc", "attn_merge", "attn_release_host_staging", "attn_set_option",
                     "attn_plan", "attn_plan_item", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
                     "attn_last_device_status")
 
@@ -58,6 +58,8 @@ def load_library() -> ctypes.CDLL:
     lib.attn_plan.restype = ci
     lib.attn_plan_item.argtypes = [ci] * 8 + [ctypes.POINTER(ci)]
     lib.attn_plan_item.restype = ci
+    lib.attn_merge.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
+    lib.attn_merge.restype = ci
     lib.attn_selftest_wait_timeout.argtypes = [ci, vp]
     lib.attn_selftest_wait_timeout.restype = ci
     lib.attn_status_str.argtypes = [ci]
@@ -170,6 +172,33 @@ def attn_plan_item(B, Hq, Hkv, Sq, Sk, D, causal, w) -> dict:
         raise AttnError(st, "attn_plan_item")
     keys = ("b", "hkv", "hq0", "hq1", "row0_0", "row0_1", "n_blocks_0", "n_blocks_1")
     return dict(zip(keys, list(out)))
+
+
+def attn_merge_status(o1, lse1, o2, lse2, o, lse, stream=None) -> int:
+    """Calls ``attn_merge`` on CUDA tensors and returns its raw status code."""
+    for name, t in (("o1", o1), ("o2", o2), ("o", o)):
+        if t.dtype != torch.bfloat16 or t.dim() != 4 or not t.is_contiguous() or t.device.type != "cuda":
+            raise ValueError(f"{name} must be a contiguous 4-D bfloat16 cuda tensor [B, Sq, Hq, D]")
+    B, Sq, Hq, D = o1.shape
+    if o2.shape != o1.shape or o.shape != o1.shape:
+        raise ValueError("inconsistent o shapes")
+    for name, t in (("lse1", lse1), ("lse2", lse2), ("lse", lse)):
+        if t.dtype != torch.float32 or not t.is_contiguous() or tuple(t.shape) != (B, Hq, Sq) or t.device.type != "cuda":
+            raise ValueError(f"{name} must be a contiguous float32 cuda tensor [B, Hq, Sq]")
+    if stream is None:
+        stream = torch.cuda.current_stream(o1.device).cuda_stream
+    with torch.cuda.device(o1.device):
+        return load_library().attn_merge(o1.data_ptr(), lse1.data_ptr(), o2.data_ptr(), lse2.data_ptr(),
+                                         o.data_ptr(), lse.data_ptr(), B, Hq, Sq, D, stream)
+
+
+def attn_merge(o1, lse1, o2, lse2, o, lse, stream=None) -> None:
+    """``attn_merge`` of the C ABI: attention over the union of two disjoint key sets from the
+    two partial results (o_i BF16 [B,Sq,Hq,D], lse_i FP32 [B,Hq,Sq]).  ``o`` may be ``o1`` or
+    ``o2``; ``lse`` must be a separate tensor."""
+    st = attn_merge_status(o1, lse1, o2, lse2, o, lse, stream)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_merge")
 
 
 def attn_selftest_wait_timeout(limit_ms: int, device=0, stream=None) -> None:

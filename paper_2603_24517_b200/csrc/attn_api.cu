@@ -8,6 +8,7 @@
 #include "../../include/attn.h"
 #include "attn_fwd_kernel.cuh"
 #include "attn_fwd_sb3.cuh"
+#include "attn_merge_kernel.cuh"
 
 namespace {
 
@@ -435,6 +436,31 @@ attn_status_t attn_set_option(const char* name, int value) {
     return ATTN_OK;
   }
   return ATTN_ERR_UNSUPPORTED;
+}
+
+attn_status_t attn_merge(const void* o1, const float* lse1, const void* o2, const float* lse2, void* o, float* lse,
+                         int B, int Hq, int Sq, int D, void* stream) {
+  if (o1 == nullptr || o2 == nullptr || o == nullptr || lse1 == nullptr || lse2 == nullptr || lse == nullptr)
+    return ATTN_ERR_NULL;
+  if (B <= 0 || Hq <= 0 || Sq <= 0 || D <= 0) return ATTN_ERR_SHAPE;
+  if (D != attn::kHeadDim) return ATTN_ERR_UNSUPPORTED;
+  const uintptr_t mask = 15;
+  if ((reinterpret_cast<uintptr_t>(o1) & mask) || (reinterpret_cast<uintptr_t>(o2) & mask) ||
+      (reinterpret_cast<uintptr_t>(o) & mask) || (reinterpret_cast<uintptr_t>(lse1) & 3) ||
+      (reinterpret_cast<uintptr_t>(lse2) & 3) || (reinterpret_cast<uintptr_t>(lse) & 3))
+    return ATTN_ERR_ALIGN;
+  if (lse == lse1 || lse == lse2) return ATTN_ERR_UNSUPPORTED;
+  attn_status_t st = ATTN_OK;
+  DeviceState* dev = device_state(&st);
+  if (dev == nullptr) return st;
+  const long long n_chunks = static_cast<long long>(B) * Sq * Hq * attn::kChunksPerRow;
+  long long blocks = (n_chunks + attn::kMergeThreads - 1) / attn::kMergeThreads;
+  const long long cap = static_cast<long long>(dev->sm_count) * 8;  // 8 resident CTAs of 256 threads per SM
+  if (blocks > cap) blocks = cap;
+  attn::attn_merge_kernel<<<static_cast<int>(blocks), attn::kMergeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint4*>(o1), lse1, static_cast<const uint4*>(o2), lse2, static_cast<uint4*>(o), lse, Hq, Sq,
+      n_chunks);
+  return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
 attn_status_t attn_selftest_wait_timeout(int limit_ms, void* stream) {

@@ -1,0 +1,76 @@
+// LSE-weighted merge of two partial attention results over disjoint key sets (HBM-bound,
+// elementwise): O = w1 O1 + w2 O2 with w_i = exp(LSE_i - LSE), LSE = log(exp(LSE1) + exp(LSE2)).
+// One thread handles one 16-byte chunk (8 BF16) of a [B, Sq, Hq, 128] row per grid-stride step, so
+// consecutive threads touch consecutive 16-byte chunks: fully coalesced 128-bit loads and stores.
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace attn {
+
+constexpr int kMergeThreads = 256;
+constexpr int kChunksPerRow = 128 * 2 / 16;  // 16-byte chunks in a 128-element BF16 row
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ uint32_t merge_pair(uint32_t a, uint32_t b, float w1, float w2) {
+  const float lo = fmaf(w1, bf16_lo(a), w2 * bf16_lo(b));
+  const float hi = fmaf(w1, bf16_hi(a), w2 * bf16_hi(b));
+  uint32_t y;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(y) : "f"(hi), "f"(lo));
+  return y;
+}
+
+constexpr int kMergeUnroll = 1;  // 16-byte chunks per thread and step (more in flight measured slower)
+
+__global__ void __launch_bounds__(kMergeThreads)
+attn_merge_kernel(const uint4* __restrict__ o1, const float* __restrict__ lse1, const uint4* __restrict__ o2,
+                  const float* __restrict__ lse2, uint4* __restrict__ o, float* __restrict__ lse, int Hq, int Sq,
+                  long long n_chunks) {
+  const long long stride = static_cast<long long>(gridDim.x) * kMergeThreads;
+  for (long long c0 = static_cast<long long>(blockIdx.x) * kMergeThreads + threadIdx.x; c0 < n_chunks;
+       c0 += stride * kMergeUnroll) {
+    uint4 x[kMergeUnroll], y[kMergeUnroll];
+    float a[kMergeUnroll], bb[kMergeUnroll];
+    long long li[kMergeUnroll];
+#pragma unroll
+    for (int u = 0; u < kMergeUnroll; ++u) {  // all loads first: kMergeUnroll x 2 x 16 bytes in flight
+      const long long c = c0 + u * stride;
+      if (c < n_chunks) {
+        const long long row = c / kChunksPerRow;  // (b * Sq + i) * Hq + h
+        const int h = static_cast<int>(row % Hq);
+        const long long t = row / Hq;
+        const int i = static_cast<int>(t % Sq);
+        const long long b = t / Sq;
+        li[u] = (b * Hq + h) * Sq + i;  // LSE is [B, Hq, Sq]
+        x[u] = __ldg(o1 + c);
+        y[u] = __ldg(o2 + c);
+        a[u] = __ldg(lse1 + li[u]);
+        bb[u] = __ldg(lse2 + li[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kMergeUnroll; ++u) {
+      const long long c = c0 + u * stride;
+      if (c < n_chunks) {
+        const float m = fmaxf(a[u], bb[u]);
+        float w1 = 0.f, w2 = 0.f, tot = -INFINITY;
+        if (m != -INFINITY) {
+          tot = m + logf(expf(a[u] - m) + expf(bb[u] - m));
+          w1 = expf(a[u] - tot);
+          w2 = expf(bb[u] - tot);
+        }
+        uint4 r;
+        r.x = merge_pair(x[u].x, y[u].x, w1, w2);
+        r.y = merge_pair(x[u].y, y[u].y, w1, w2);
+        r.z = merge_pair(x[u].z, y[u].z, w1, w2);
+        r.w = merge_pair(x[u].w, y[u].w, w1, w2);
+        o[c] = r;
+        if ((c % kChunksPerRow) == 0) lse[li[u]] = tot;
+      }
+    }
+  }
+}
+
+}  // namespace attn

@@ -260,3 +260,43 @@ def test_bad_arguments_are_rejected():
     q, k, v = (bf16_bits(t) for t in make_qkv(1, 2, 2, 4, 4, 8, seed=141))
     with pytest.raises(ValueError):
         orc.attention_rows(q, k, v, False, 1.0, np.array([[0, 0, 4]], dtype=np.int32))
+
+
+def _f32_to_bits(x):
+    return to_bits(x)
+
+
+def test_merge_of_exact_halves_reproduces_the_whole():
+    """Pins attn_oracle_merge: feed it partial results that are exactly representable (BF16 O parts
+    from one-hot softmaxes) and compare with the attention over all keys."""
+    # one query, D = 2; part 1 = key A only, part 2 = key B only: O_i = v_i exactly, LSE_i = s_i
+    va, vb = np.array([1.0, -2.0]), np.array([0.5, 4.0])
+    sa, sb = 1.25, -0.75          # exactly representable in fp32
+    o, lse = orc.merge(to_bits(va.reshape(1, 2)), np.array([sa], np.float32),
+                       to_bits(vb.reshape(1, 2)), np.array([sb], np.float32))
+    wa = 1.0 / (1.0 + math.exp(sb - sa))
+    np.testing.assert_allclose(o[0], wa * va + (1 - wa) * vb, atol=1e-15)
+    assert lse[0] == pytest.approx(math.log(math.exp(sa) + math.exp(sb)), abs=1e-15)
+
+
+def test_merge_special_cases():
+    o1 = rand_bits((5, 8), 200)
+    o2 = rand_bits((5, 8), 201)
+    l1 = np.linspace(-3, 3, 5).astype(np.float32)
+    # an empty second part changes nothing
+    o, lse = orc.merge(o1, l1, o2, np.full(5, -np.inf, np.float32))
+    np.testing.assert_array_equal(o, bits_to_float64(o1))
+    np.testing.assert_array_equal(lse, l1.astype(np.float64))
+    # equal LSEs: plain average, LSE + log 2
+    o, lse = orc.merge(o1, l1, o2, l1)
+    np.testing.assert_allclose(o, 0.5 * (bits_to_float64(o1) + bits_to_float64(o2)), atol=1e-15)
+    np.testing.assert_allclose(lse, l1.astype(np.float64) + math.log(2.0), atol=1e-15)
+    # symmetric in its two parts
+    l2 = l1[::-1].copy()
+    oa, la = orc.merge(o1, l1, o2, l2)
+    ob, lb = orc.merge(o2, l2, o1, l1)
+    np.testing.assert_allclose(oa, ob, atol=1e-15)
+    np.testing.assert_allclose(la, lb, atol=1e-15)
+    # both empty
+    o, lse = orc.merge(o1, np.full(5, -np.inf, np.float32), o2, np.full(5, -np.inf, np.float32))
+    assert np.all(o == 0) and np.all(lse == -np.inf)
