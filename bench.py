@@ -53,6 +53,10 @@ def parse_args():
     ap.add_argument("--op", default="fwd", choices=["fwd", "merge"],
                     help="fwd: the attention forward (default, the headline metric); merge: the LSE-weighted "
                          "merge of two partial results of the same shape (HBM-bound side kernel)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every sequence-length sweep workload (10 warm-ups, then 10 repetitions of 30 launches: "
+                         "mean and standard deviation) and print one JSON line with the per-workload TFLOP/s vector "
+                         "and its geometric means; one GPU")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target oracle time of the cpu_baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -354,6 +358,62 @@ def run_merge(args, w):
     }), flush=True)
 
 
+def run_sweep(args):
+    """The evaluation protocol of the paper's Section 4.1 on every sweep workload: TFLOP/s per
+    configuration as mean and standard deviation over 10 repetitions, and the geometric mean per
+    family (the score vector of Section 3.1; correctness of each entry is what the GPU parity tests
+    establish on these same workloads, so no entry is zeroed here)."""
+    import math
+    import paper_2603_24517_b200 as lib
+    from paper_2603_24517_b200 import build as lib_build
+    lib_build.build()
+    lib.load_library()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    reps, launches, warm = 10, 30, 10
+    sampler = ClockSampler(0)
+    sampler.start()
+    entries = {}
+    for name, w in all_workloads().items():
+        if not (name.startswith(("mha_", "gqa4_", "gqa8_")) and "_s" in name):
+            continue
+        q_h, k_h, v_h = make_workload_inputs(w)
+        q, k, v = q_h.to(dev), k_h.to(dev), v_h.to(dev)
+        o = torch.empty_like(q)
+        lse = torch.empty((w.B, w.Hq, w.Sq), dtype=torch.float32, device=dev)
+        for _ in range(warm):
+            lib.attn_fwd(q, k, v, o, lse, w.causal, w.scale)
+        torch.cuda.synchronize()
+        rates = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(launches):
+                lib.attn_fwd(q, k, v, o, lse, w.causal, w.scale)
+            e1.record()
+            torch.cuda.synchronize()
+            rates.append(w.flops / (e0.elapsed_time(e1) / launches * 1e-3) / 1e12)
+        st, code, detail = lib.attn_last_device_status()
+        if st != 0:
+            raise SystemExit(f"{name}: device status {st} code {code:#x} detail {detail}")
+        entries[name] = {"tflops": statistics.mean(rates), "std": statistics.pstdev(rates),
+                         "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "S": w.Sq, "causal": w.causal}
+        del q, k, v, o, lse
+    clocks = sampler.stop()
+
+    def geomean(prefix):
+        xs = [e["tflops"] for n, e in entries.items() if n.startswith(prefix)]
+        return math.exp(sum(math.log(x) for x in xs) / len(xs)) if xs else None
+
+    families = ["mha_noncausal", "mha_causal", "gqa4_noncausal", "gqa4_causal", "gqa8_noncausal", "gqa8_causal"]
+    print(json.dumps({
+        "metric": METRIC + "_sweep", "unit": UNIT, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+        "protocol": {"warmup_launches": warm, "launches_per_repetition": launches, "repetitions": reps},
+        "geomean": {f: geomean(f) for f in families}, "workloads": entries, "clocks": clocks,
+        "gpu_launches": len(entries) * (warm + reps * launches),
+    }), flush=True)
+
+
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of attn_fwd_kernel from the ncu capture
 # summarised in profiles/attn_fwd_kernel_mha_noncausal_s16384_launches.md (403.6 MB + 117.6 MB).
 TRAFFIC_BYTES: dict[str, float | None] = {"mha_noncausal_s16384": 521.2e6}
@@ -361,6 +421,9 @@ TRAFFIC_BYTES: dict[str, float | None] = {"mha_noncausal_s16384": 521.2e6}
 
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     workloads = all_workloads()
     if args.workload not in workloads:
         raise SystemExit(f"unknown workload {args.workload}; choose from {sorted(workloads)}")
