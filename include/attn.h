@@ -28,7 +28,7 @@ typedef enum {
   ATTN_OK = 0,
   ATTN_ERR_NULL = 1,        /* a required pointer is NULL */
   ATTN_ERR_SHAPE = 2,       /* a dimension is <= 0, or Hq is not a multiple of Hkv */
-  ATTN_ERR_UNSUPPORTED = 3, /* D != 128; causal with Sq > Sk; scale not finite or <= 0 */
+  ATTN_ERR_UNSUPPORTED = 3, /* D != 128; scale not finite or <= 0; sizes beyond the index range */
   ATTN_ERR_ALIGN = 4,       /* q, k, v or o not 16-byte aligned; lse not 4-byte aligned */
   ATTN_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed (descriptor, launch, copy) */
   ATTN_ERR_ARCH = 6,        /* the current device is not compute capability 10.x */
@@ -54,7 +54,8 @@ typedef enum {
  *                       128-row tile); Hq % Hkv == 0
  *   D        must be 128
  *   causal   0: every key is visible.  non-zero: key j is visible to query i iff
- *            j <= i + (Sk - Sq)  (lower-triangular when Sq == Sk); requires Sq <= Sk
+ *            j <= i + (Sk - Sq)  (lower-triangular when Sq == Sk).  With Sq > Sk the
+ *            first Sq - Sk rows see no key: their o is 0 and their lse is -infinity
  *   scale    multiplies Q K^T; finite and > 0 (callers normally pass 1/sqrt(D))
  *   stream   cudaStream_t (NULL = default stream)
  *

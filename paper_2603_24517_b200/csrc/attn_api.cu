@@ -113,7 +113,6 @@ attn_status_t check_args(const void* q, const void* k, const void* v, void* o, c
   if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || D <= 0) return ATTN_ERR_SHAPE;
   if (Hq % Hkv != 0) return ATTN_ERR_SHAPE;
   if (D != attn::kHeadDim) return ATTN_ERR_UNSUPPORTED;
-  if (causal && Sq > Sk) return ATTN_ERR_UNSUPPORTED;
   if (!std::isfinite(scale) || !(scale > 0.f)) return ATTN_ERR_UNSUPPORTED;
   // sizes the 32-bit tile arithmetic and the TMA coordinates can hold
   if (static_cast<long long>(B) * Hq * ((Sq + 127) / 128) > 0x3fffffffLL) return ATTN_ERR_UNSUPPORTED;

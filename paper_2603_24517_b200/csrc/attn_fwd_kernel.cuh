@@ -145,7 +145,10 @@ __host__ __device__ __forceinline__ void decode_work(const FwdParams& p, int w, 
       wk.n[s] = 0;
     } else if (p.causal) {
       const int row_end = wk.row0[s] + kTile < p.Sq ? wk.row0[s] + kTile : p.Sq;
-      const int need = (row_end - 1 + p.off) / kTile + 1;
+      // a tile none of whose rows sees a key (Sq > Sk) still visits one, fully masked, block, so
+      // that its O = 0 and LSE = -inf are produced by the ordinary path
+      const int last_key = row_end - 1 + p.off;
+      const int need = last_key < 0 ? 1 : last_key / kTile + 1;
       wk.n[s] = need < p.n_kb ? need : p.n_kb;
     } else {
       wk.n[s] = p.n_kb;
@@ -556,7 +559,9 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
     bool ok = mbar_wait(&bars.l_empty[s], (l_cnt & 1) ^ 1, ctx, kRoleSoftmax | kBarLEmpty);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) return;
-    stats[row_in_tile] = l;
+    // a row without any visible key (causal, Sq > Sk) has the sum 0 by definition; its masked
+    // scores may have left denormal-sized terms in l
+    stats[row_in_tile] = row_limit > 0 ? l : 0.f;
     stats[kTile + row_in_tile] = m_used;
     mbar_arrive(&bars.l_full[s]);
     ++l_cnt;
@@ -595,7 +600,7 @@ __device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers
       }
       ++cnt[s];
       tc_fence_after_sync();
-      const float inv_l = 1.0f / l;
+      const float inv_l = l > 0.f ? 1.0f / l : 0.f;  // l = 0: a row without visible keys, O = 0 and LSE = -inf
       // the previous TMA store must have finished reading the staging tile
       ok = mbar_wait(&bars.stg_empty[0], (stg_cnt & 1) ^ 1, ctx, kRoleEpilogue | kBarStgEmpty);
       ok = __all_sync(0xffffffffu, ok);

@@ -82,7 +82,8 @@ __host__ __device__ __forceinline__ void decode_item(const FwdParams& p, int w, 
   it.row0 = qt * kTile;
   if (p.causal) {
     const int row_end = it.row0 + kTile < p.Sq ? it.row0 + kTile : p.Sq;
-    const int need = (row_end - 1 + p.off) / kTile + 1;
+    const int last_key = row_end - 1 + p.off;  // < 0: no row of the tile sees a key; one masked block is visited
+    const int need = last_key < 0 ? 1 : last_key / kTile + 1;
     it.n = need < p.n_kb ? need : p.n_kb;
   } else {
     it.n = p.n_kb;
@@ -420,7 +421,7 @@ __device__ __forceinline__ void role_softmax3(const FwdParams& p, const Bars3& b
     }
     // hand this group's partial sum and its reference to the epilogue warps
     if (!mbar_wait_warp(&bars.l_empty[0], (item_cnt & 1) ^ 1, ctx, kRoleSoftmax | kBarLEmpty)) return;
-    stats[row_in_tile] = has ? l : 0.f;
+    stats[row_in_tile] = (has && row_limit > 0) ? l : 0.f;  // no visible key (causal, Sq > Sk): the sum is 0
     stats[kTile + row_in_tile] = m_last;
     mbar_arrive(&bars.l_full[0]);
     base0 += blocks_in_buffer(n, 0);
@@ -456,7 +457,7 @@ __device__ __forceinline__ void role_epilogue3(const FwdParams& p, const Bars3& 
     if (l1 > 0.f) l_row += l1 * ex2_approx((m1 - m_fin) * c);
     if (!mbar_wait_warp(&bars.o_full[0], item_cnt & 1, ctx, kRoleEpilogue | kBarOFull)) return;
     tc_fence_after_sync();
-    const float inv_l = 1.0f / l_row;
+    const float inv_l = l_row > 0.f ? 1.0f / l_row : 0.f;  // a row without visible keys: O = 0, LSE = -inf
     uint8_t* stage = smem + kSmemQ3;
 #pragma unroll
     for (int cc = 0; cc < 4; ++cc) {

@@ -54,6 +54,15 @@ def run_gpu(q, k, v, causal, scale, want_lse=True, stream=None):
     return o.cpu(), (None if lse is None else lse.cpu())
 
 
+def lse_distance(l64, lse_ref):
+    """max |dLSE| over the rows that see a key; rows that see none (causal, Sq > Sk) must be
+    -inf on both sides."""
+    empty = np.isneginf(lse_ref)
+    assert np.array_equal(np.isneginf(l64), empty), "rows without visible keys must have LSE = -inf"
+    assert np.isfinite(l64[~empty]).all()
+    return np.abs(l64[~empty] - lse_ref[~empty]).max() if (~empty).any() else 0.0
+
+
 def check_full(q, k, v, causal, scale, o, lse):
     o_ref, lse_ref = orc.attention_full(bf16_bits(q), bf16_bits(k), bf16_bits(v), causal, scale)
     o64 = bits_to_float64(bf16_bits(o))
@@ -63,7 +72,7 @@ def check_full(q, k, v, causal, scale, o, lse):
     if lse is not None:
         l64 = lse.numpy().astype(np.float64)
         assert not np.isnan(l64).any()
-        d_l = np.abs(l64 - lse_ref).max()
+        d_l = lse_distance(l64, lse_ref)
         assert d_l <= TOL_LSE, f"max|dLSE| = {d_l}"
 
 
@@ -72,7 +81,7 @@ def check_rows(q, k, v, causal, scale, o, lse, rows):
     o64 = bits_to_float64(bf16_bits(o))[rows[:, 0], rows[:, 2], rows[:, 1]]
     l64 = lse.numpy().astype(np.float64)[rows[:, 0], rows[:, 1], rows[:, 2]]
     assert not np.isnan(o64).any() and not np.isnan(l64).any()
-    d_o, d_l = np.abs(o64 - o_ref).max(), np.abs(l64 - lse_ref).max()
+    d_o, d_l = np.abs(o64 - o_ref).max(), lse_distance(l64, lse_ref)
     assert d_o <= TOL_O, f"max|dO| = {d_o}"
     assert d_l <= TOL_LSE, f"max|dLSE| = {d_l}"
 
@@ -99,6 +108,10 @@ SMALL = [
     (1, 8, 1, 384, 384, True),        # group 8
     (5, 2, 2, 200, 136, False),
     (1, 4, 4, 1280, 1280, True),      # more K/V blocks than ring slots, several items per CTA
+    (1, 2, 2, 384, 128, True),        # Sq > Sk: the first 256 rows (two whole tiles) see no key
+    (2, 4, 2, 300, 77, True),         # Sq > Sk, ragged: rows 0..222 see no key, GQA pairs row tiles
+    (1, 8, 2, 200, 130, True),        # Sq > Sk with stages pairing query heads
+    (1, 1, 1, 129, 1, True),          # only the last row sees the single key
 ]
 
 
@@ -237,8 +250,8 @@ def test_expired_wait_is_reported_and_the_device_stays_usable():
 def test_error_statuses_on_device_tensors():
     q, k, v = (t.cuda() for t in make_qkv(1, 2, 2, 256, 128, 128, seed=7800))
     o = torch.empty_like(q)
-    assert lib.attn_fwd_status(q, k, v, o, None, True, SCALE) == 3     # causal with Sq > Sk
     assert lib.attn_fwd_status(q, k, v, o, None, False, -1.0) == 3
+    assert lib.attn_fwd_status(q, k, v, o, None, False, float("nan")) == 3
     assert lib.attn_fwd_status(q, k, v, o, None, False, SCALE) == 0
     torch.cuda.synchronize()
 

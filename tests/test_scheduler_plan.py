@@ -27,6 +27,8 @@ def visible_blocks_brute(row0, Sq, Sk, causal):
     if not causal:
         return math.ceil(Sk / TILE)
     last_key = max(min(Sk - 1, i + Sk - Sq) for i in rows)
+    if last_key < 0:  # Sq > Sk: no row of the tile sees a key; one masked block is still visited
+        return 1      # so that the tile's O = 0 and LSE = -inf get written
     return last_key // TILE + 1
 
 
@@ -35,6 +37,7 @@ CASES = [
     (1, 8, 2, 300, 300, True), (1, 8, 2, 300, 700, False), (2, 32, 8, 1024, 1024, True),
     (1, 32, 4, 640, 640, True), (1, 6, 2, 130, 130, True), (1, 5, 5, 1, 1, False),
     (3, 4, 4, 129, 1000, True), (1, 16, 16, 16384, 16384, True),
+    (1, 2, 2, 640, 128, True), (2, 4, 2, 700, 77, True), (1, 8, 2, 513, 300, True),  # Sq > Sk
 ]
 
 
@@ -118,6 +121,6 @@ def test_plan_rejects_bad_problems():
     with pytest.raises(lib.AttnError):
         lib.attn_plan(1, 3, 2, 128, 128, 128, False, 148)
     with pytest.raises(lib.AttnError):
-        lib.attn_plan(1, 2, 2, 256, 128, 128, True, 148)
+        lib.attn_plan(1, 2, 2, 256, 128, 64, True, 148)
     with pytest.raises(lib.AttnError):
         lib.attn_plan_item(1, 2, 2, 128, 128, 128, False, 99)
