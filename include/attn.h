@@ -71,6 +71,33 @@ attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, flo
                        int causal, float scale, void* stream);
 
 /*
+ * attn_fwd_strided -- attn_fwd on strided views (the paper states no memory layout; this
+ * entry point takes any layout whose head dimension is contiguous).
+ *
+ * Same operation, arithmetic, result and rules as attn_fwd.  q, k, v, o are indexed as
+ *   x[b, s, h, d] = base[b * strides[0] + s * strides[1] + h * strides[2] + d]
+ * with x_strides = {batch, sequence, head} strides in ELEMENTS (host arrays of 3, read
+ * during the call only).  Examples: a [B, H, S, D] buffer is {H*S*D, D, S*D}; the q slice of
+ * a packed [B, S, 3, H, D] projection is {3*S*H*D, 3*H*D, D} with base + 0; the keys
+ * s0 .. s0+n of a longer sequence are the same strides with base + s0 * strides[1] and
+ * Sk = n (attn_merge combines the partial results of disjoint key ranges).  lse is always
+ * contiguous [B, Hq, Sq].
+ *
+ * Every stride must be positive and a multiple of 8 elements (16 bytes: the tiles move by
+ * TMA), the sequence and head strides at least 128, all below 2^39 elements; an axis of
+ * extent 1 still needs a legal value.  Errors: ATTN_ERR_NULL for a missing stride array,
+ * ATTN_ERR_SHAPE for a stride <= 0 or < 128 where rows would overlap, ATTN_ERR_ALIGN for a
+ * stride that is not a multiple of 8, ATTN_ERR_UNSUPPORTED beyond the range, and
+ * ATTN_ERR_CUDA if the driver rejects the resulting descriptor.  Rows addressed by
+ * different (b, s, h) of o must not overlap; the inputs may overlap each other freely.
+ */
+attn_status_t attn_fwd_strided(const void* q, const void* k, const void* v, void* o, float* lse,
+                               int B, int Hq, int Hkv, int Sq, int Sk, int D,
+                               const long long* q_strides, const long long* k_strides,
+                               const long long* v_strides, const long long* o_strides,
+                               int causal, float scale, void* stream);
+
+/*
  * attn_fwd_host -- the same operation on HOST buffers (same layouts).  Copies q, k, v
  * to library-owned device staging buffers (grown on demand, kept for later calls),
  * runs attn_fwd, copies o and lse (if not NULL) back and synchronises `stream` before

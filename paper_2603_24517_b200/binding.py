@@ -20,7 +20,7 @@ STATUS_NAMES = {
     0: "ATTN_OK", 1: "ATTN_ERR_NULL", 2: "ATTN_ERR_SHAPE", 3: "ATTN_ERR_UNSUPPORTED", 4: "ATTN_ERR_ALIGN",
     5: "ATTN_ERR_CUDA", 6: "ATTN_ERR_ARCH", 7: "ATTN_ERR_TIMEOUT", 8: "ATTN_ERR_TOO_LARGE",
 }
-EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_host", "attn_fwd_noalloc", "attn_merge", "attn_release_host_staging", "attn_set_option",
+EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_strided", "attn_fwd_host", "attn_fwd_noalloc", "attn_merge", "attn_release_host_staging", "attn_set_option",
                     "attn_plan", "attn_plan_item", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
                     "attn_last_device_status")
 
@@ -49,6 +49,9 @@ def load_library() -> ctypes.CDLL:
     lib.attn_fwd_host.argtypes = fwd_args
     lib.attn_fwd_host.restype = ci
     lib.attn_fwd_noalloc.argtypes = fwd_args
+    ll3 = ctypes.POINTER(ctypes.c_longlong)
+    lib.attn_fwd_strided.argtypes = fwd_args[:11] + [ll3, ll3, ll3, ll3] + fwd_args[11:]
+    lib.attn_fwd_strided.restype = ci
     lib.attn_fwd_noalloc.restype = ci
     lib.attn_release_host_staging.argtypes = []
     lib.attn_release_host_staging.restype = ci
@@ -104,6 +107,46 @@ def attn_fwd(q, k, v, o, lse, causal: bool, scale: float, stream=None) -> None:
     st = attn_fwd_status(q, k, v, o, lse, causal, scale, stream)
     if st != ATTN_OK:
         raise AttnError(st, "attn_fwd")
+
+
+def _strides3(t):
+    """Element strides of the (batch, sequence, head) axes of a [B, S, H, D] tensor as a C array.
+    An axis of extent 1 is never stepped along, so it gets the stride a contiguous tensor would
+    have (torch may report anything there)."""
+    _, S, H, D = t.shape
+    dense = (S * H * D, H * D, D)
+    vals = [dense[i] if t.shape[i] == 1 else t.stride(i) for i in range(3)]
+    return (ctypes.c_longlong * 3)(*vals)
+
+
+def attn_fwd_strided_status(q, k, v, o, lse, causal: bool, scale: float, stream=None) -> int:
+    """Calls ``attn_fwd_strided`` on CUDA tensors of shape [B, S, H, D] with arbitrary batch,
+    sequence and head strides (the head dimension must be contiguous); returns the raw status."""
+    for name, t in (("q", q), ("k", k), ("v", v), ("o", o)):
+        if t.dtype != torch.bfloat16 or t.dim() != 4 or t.stride(3) != 1 or t.device.type != "cuda":
+            raise ValueError(f"{name} must be a 4-D bfloat16 cuda tensor [B, S, H, D] with a contiguous last axis")
+    B, Sq, Hq, D = q.shape
+    Bk, Sk, Hkv, Dk = k.shape
+    if v.shape != k.shape or o.shape != q.shape or Bk != B or Dk != D:
+        raise ValueError("inconsistent q/k/v/o shapes")
+    if lse is not None and (lse.dtype != torch.float32 or not lse.is_contiguous()
+                            or tuple(lse.shape) != (B, Hq, Sq) or lse.device.type != "cuda"):
+        raise ValueError("lse must be a contiguous float32 tensor [B, Hq, Sq]")
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        return load_library().attn_fwd_strided(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                               None if lse is None else lse.data_ptr(),
+                                               B, Hq, Hkv, Sq, Sk, D, _strides3(q), _strides3(k), _strides3(v),
+                                               _strides3(o), int(bool(causal)), float(scale), stream)
+
+
+def attn_fwd_strided(q, k, v, o, lse, causal: bool, scale: float, stream=None) -> None:
+    """``attn_fwd_strided`` of the C ABI: ``attn_fwd`` on views -- a [B, H, S, D] buffer seen as
+    [B, S, H, D], slices of a packed QKV projection, a key range of a longer sequence."""
+    st = attn_fwd_strided_status(q, k, v, o, lse, causal, scale, stream)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_fwd_strided")
 
 
 def attn_fwd_noalloc_status(q, k, v, o, lse, causal: bool, scale: float, stream=None) -> int:

@@ -93,13 +93,22 @@ DeviceState* device_state(attn_status_t* st) {
   return &d;
 }
 
-// [B, S, H, 128] BF16 tensor seen as 4-D (D, H, S, B); box = 64 elements x 1 head x 128 rows,
-// 128-byte swizzle, out-of-range rows read as zero and are clipped on store.
-bool make_tensor_map(CUtensorMap* tm, const void* base, int B, int S, int H) {
+// Element strides of the (batch, sequence, head) axes of a [B, S, H, 128] BF16 tensor; the head
+// dimension is contiguous.
+struct Strides3 {
+  long long b, s, h;
+};
+Strides3 contiguous_strides(int S, int H) {
+  return Strides3{static_cast<long long>(S) * H * 128, static_cast<long long>(H) * 128, 128};
+}
+
+// BF16 tensor seen as 4-D (D, H, S, B) with the given element strides; box = 64 elements x 1 head
+// x 128 rows, 128-byte swizzle, out-of-range rows read as zero and are clipped on store.
+bool make_tensor_map(CUtensorMap* tm, const void* base, int B, int S, int H, Strides3 st) {
   const cuuint64_t dims[4] = {128, static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(S),
                               static_cast<cuuint64_t>(B)};
-  const cuuint64_t strides[3] = {128ull * 2, static_cast<cuuint64_t>(H) * 128 * 2,
-                                 static_cast<cuuint64_t>(S) * H * 128 * 2};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(st.h) * 2, static_cast<cuuint64_t>(st.s) * 2,
+                                 static_cast<cuuint64_t>(st.b) * 2};
   const cuuint32_t box[4] = {64, 1, 128, 1};
   const cuuint32_t elem_strides[4] = {1, 1, 1, 1};
   return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
@@ -246,16 +255,34 @@ attn_status_t attn_plan_item(int B, int Hq, int Hkv, int Sq, int Sk, int D, int 
   return ATTN_OK;
 }
 
-attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
-                       int Sq, int Sk, int D, int causal, float scale, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// A stride the TMA engine accepts: positive, a multiple of 8 elements (16 bytes), below 2^40
+// bytes; axes of extent 1 are never stepped along, but the descriptor still wants a legal value.
+attn_status_t check_strides(const long long* s) {
+  if (s == nullptr) return ATTN_ERR_NULL;
+  for (int i = 0; i < 3; ++i) {
+    if (s[i] <= 0) return ATTN_ERR_SHAPE;
+    if (s[i] % 8 != 0) return ATTN_ERR_ALIGN;
+    if (s[i] >= (1ll << 39)) return ATTN_ERR_UNSUPPORTED;
+  }
+  if (s[1] < 128 || s[2] < 128) return ATTN_ERR_SHAPE;  // rows of 128 contiguous elements must not overlap
+  return ATTN_OK;
+}
+
+attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
+                         int Sq, int Sk, int D, Strides3 sq, Strides3 sk, Strides3 sv, Strides3 so, int causal,
+                         float scale, void* stream) {
   attn_status_t st = check_args(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, scale, true);
   if (st != ATTN_OK) return st;
   DeviceState* dev = device_state(&st);
   if (dev == nullptr) return st;
 
   CUtensorMap tm_q, tm_k, tm_v, tm_o;
-  if (!make_tensor_map(&tm_q, q, B, Sq, Hq) || !make_tensor_map(&tm_k, k, B, Sk, Hkv) ||
-      !make_tensor_map(&tm_v, v, B, Sk, Hkv) || !make_tensor_map(&tm_o, o, B, Sq, Hq))
+  if (!make_tensor_map(&tm_q, q, B, Sq, Hq, sq) || !make_tensor_map(&tm_k, k, B, Sk, Hkv, sk) ||
+      !make_tensor_map(&tm_v, v, B, Sk, Hkv, sv) || !make_tensor_map(&tm_o, o, B, Sq, Hq, so))
     return ATTN_ERR_CUDA;
 
   FwdParams p;
@@ -272,6 +299,31 @@ attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, flo
     if (cudaMemsetAsync(p.counter, 0, sizeof(unsigned int), s) != cudaSuccess) return ATTN_ERR_CUDA;
   }
   return launch_fwd(tm_q, tm_k, tm_v, tm_o, p, grid, s) == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+attn_status_t attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
+                       int Sq, int Sk, int D, int causal, float scale, void* stream) {
+  return fwd_device(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, contiguous_strides(Sq, Hq), contiguous_strides(Sk, Hkv),
+                    contiguous_strides(Sk, Hkv), contiguous_strides(Sq, Hq), causal, scale, stream);
+}
+
+attn_status_t attn_fwd_strided(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq,
+                               int Hkv, int Sq, int Sk, int D, const long long* q_strides,
+                               const long long* k_strides, const long long* v_strides, const long long* o_strides,
+                               int causal, float scale, void* stream) {
+  const long long* all[4] = {q_strides, k_strides, v_strides, o_strides};
+  for (const long long* s : all) {
+    const attn_status_t st = check_strides(s);
+    if (st != ATTN_OK) return st;
+  }
+  return fwd_device(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, Strides3{q_strides[0], q_strides[1], q_strides[2]},
+                    Strides3{k_strides[0], k_strides[1], k_strides[2]},
+                    Strides3{v_strides[0], v_strides[1], v_strides[2]},
+                    Strides3{o_strides[0], o_strides[1], o_strides[2]}, causal, scale, stream);
 }
 
 attn_status_t attn_fwd_host(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq,
@@ -372,8 +424,10 @@ attn_status_t attn_fwd_noalloc(const void* q, const void* k, const void* v, void
   if (st != ATTN_OK) return st;
 
   CUtensorMap tm_q, tm_k, tm_v, tm_o;
-  if (!make_tensor_map(&tm_q, q, B, Sq, Hq) || !make_tensor_map(&tm_k, k, B, Sk, Hkv) ||
-      !make_tensor_map(&tm_v, v, B, Sk, Hkv) || !make_tensor_map(&tm_o, o, B, Sq, Hq))
+  if (!make_tensor_map(&tm_q, q, B, Sq, Hq, contiguous_strides(Sq, Hq)) ||
+      !make_tensor_map(&tm_k, k, B, Sk, Hkv, contiguous_strides(Sk, Hkv)) ||
+      !make_tensor_map(&tm_v, v, B, Sk, Hkv, contiguous_strides(Sk, Hkv)) ||
+      !make_tensor_map(&tm_o, o, B, Sq, Hq, contiguous_strides(Sq, Hq)))
     return ATTN_ERR_CUDA;
 
   FwdParams p;

@@ -89,3 +89,18 @@ def test_missing_library_is_loud(monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libattn_b200.so"))
     with pytest.raises(ImportError):
         binding.load_library()
+
+
+def test_stride_errors_need_no_device(cdll):
+    import ctypes
+    arr = lambda *v: (ctypes.c_longlong * 3)(*v)
+    ok = arr(128 * 2 * 128, 2 * 128, 128)
+
+    def call(qs=ok, ks=ok, vs=ok, os_=ok):
+        return cdll.attn_fwd_strided(16, 16, 16, 16, None, 1, 2, 2, 128, 128, 128, qs, ks, vs, os_, 0, 0.1, None)
+
+    assert call(qs=None) == 1                      # ATTN_ERR_NULL
+    assert call(ks=arr(0, 256, 128)) == 2          # ATTN_ERR_SHAPE: stride <= 0
+    assert call(vs=arr(32768, 64, 128)) == 2       # rows of 128 elements would overlap
+    assert call(os_=arr(32768, 260, 128)) == 4     # ATTN_ERR_ALIGN: not a multiple of 8 elements
+    assert call(qs=arr(1 << 40, 256, 128)) == 3    # ATTN_ERR_UNSUPPORTED: beyond the descriptor's range
