@@ -100,9 +100,16 @@ attn_status_t attn_fwd_strided(const void* q, const void* k, const void* v, void
 /*
  * attn_fwd_host -- the same operation on HOST buffers (same layouts).  Copies q, k, v
  * to library-owned device staging buffers (grown on demand, kept for later calls),
- * runs attn_fwd, copies o and lse (if not NULL) back and synchronises `stream` before
- * returning.  Pinned host memory makes the copies asynchronous with respect to the
- * host; pageable memory works too.  Not re-entrant: one call at a time per process.
+ * runs the forward, copies o and lse (if not NULL) back and synchronises `stream` before
+ * returning; the work starts after whatever is already queued on `stream`.
+ * Query rows are independent, so by default the call is pipelined: chunks of whole
+ * 256-row work items (about one wave of CTAs each) are uploaded, computed (one strided
+ * launch per chunk) and downloaded on three library-owned streams, so that host-to-device
+ * copies, kernels and device-to-host copies overlap; under the causal mask a chunk waits
+ * only for the keys its rows can see.  Results are bit-identical to attn_fwd on the same
+ * data.  Option "host_pipeline" = 0 selects the plain copy / launch / copy sequence (also
+ * used for causal problems with Sq > Sk).  The overlap needs pinned host memory; pageable
+ * memory works, serialised by the driver.  Not re-entrant: one call at a time per process.
  */
 attn_status_t attn_fwd_host(const void* q, const void* k, const void* v, void* o, float* lse,
                             int B, int Hq, int Hkv, int Sq, int Sk, int D,
@@ -159,6 +166,8 @@ attn_status_t attn_release_host_staging(void);
  *   "overlap_epilogue"  1 (default) = a query stage is normalised and stored as soon as its own
  *                 last P V has completed, overlapping the other stage's (Section 5.2);
  *                 0 = only after both stages' last P V ("kernel" = 0 only)
+ *   "host_pipeline"  1 (default) = attn_fwd_host overlaps upload, compute and download in row
+ *                 chunks; 0 = one upload, one launch, one download
  *   "kernel"      0 = dual query stage: a CTA runs two 128-row query tiles against one stream
  *                     of K/V tiles, one score buffer each (default)
  *                 1 = triple score buffer: a CTA runs one query tile with three score tiles

@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "../../include/attn.h"
 #include "attn_fwd_kernel.cuh"
@@ -31,6 +32,9 @@ struct DeviceState {
   // attn_fwd_host staging
   void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   size_t stage_bytes[5] = {0, 0, 0, 0, 0};
+  // attn_fwd_host pipeline: upload, compute and download streams and a pool of events
+  cudaStream_t pipe[3] = {nullptr, nullptr, nullptr};
+  std::vector<cudaEvent_t> events;
 };
 
 std::mutex g_mutex;
@@ -42,6 +46,7 @@ std::atomic<int> g_opt_kernel{0};  // 0: dual query stage, 1: triple score buffe
 std::atomic<int> g_opt_rescale_threshold{8};
 std::atomic<int> g_opt_split_p{1};
 std::atomic<int> g_opt_overlap_epilogue{1};
+std::atomic<int> g_opt_host_pipeline{1};
 
 // Per-device one-time set-up: architecture check, kernel attribute, scheduler counters and
 // status word.  Returns the state or nullptr (with *st set).
@@ -301,6 +306,95 @@ attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, f
   return launch_fwd(tm_q, tm_k, tm_v, tm_o, p, grid, s) == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
+// attn_fwd_host as a three-stream pipeline.  Query rows are independent, so the problem is cut
+// into chunks of whole 256-row work items, about one wave of CTAs each; chunk c's kernel runs
+// while chunk c+1's rows (and, under the causal mask, only the keys that chunk c+1 newly needs)
+// are uploaded and chunk c-1's output is downloaded, on separate copy engines.  Each chunk is
+// one strided launch on views of the staging buffers; its LSE block is written compactly and
+// scattered into the caller's [B, Hq, Sq] array by a 2-D copy.
+attn_status_t host_pipeline(DeviceState* dev, const void* q, const void* k, const void* v, void* o, float* lse,
+                            int B, int Hq, int Hkv, int Sq, int Sk, int causal, float scale, cudaStream_t user) {
+  for (int i = 0; i < 3; ++i) {
+    if (dev->pipe[i] == nullptr &&
+        cudaStreamCreateWithFlags(&dev->pipe[i], cudaStreamNonBlocking) != cudaSuccess)
+      return ATTN_ERR_CUDA;
+  }
+  const cudaStream_t s_up = dev->pipe[0], s_run = dev->pipe[1], s_down = dev->pipe[2];
+  size_t next_event = 0;
+  auto event = [&]() -> cudaEvent_t {
+    if (next_event == dev->events.size()) {
+      cudaEvent_t e = nullptr;
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      dev->events.push_back(e);
+    }
+    return dev->events[next_event++];
+  };
+  bool ok = true;
+  auto after = [&](cudaStream_t waiter, cudaStream_t signaller) {  // waiter continues after signaller's work so far
+    cudaEvent_t e = event();
+    ok = ok && e != nullptr && cudaEventRecord(e, signaller) == cudaSuccess &&
+         cudaStreamWaitEvent(waiter, e, 0) == cudaSuccess;
+  };
+  // the pipeline starts after whatever the caller has queued on its stream
+  after(s_up, user);
+  after(s_run, user);
+  after(s_down, user);
+
+  const int D = attn::kHeadDim;
+  const int off = Sk - Sq;  // >= 0 here
+  const int waves = dev->sm_count / Hq > 0 ? dev->sm_count / Hq : 1;  // 256-row items of all heads per wave
+  int chunk_rows = 256 * waves;
+  if ((Sq + chunk_rows - 1) / chunk_rows > 64) chunk_rows = ((Sq + 63) / 64 + 255) / 256 * 256;
+  const uint8_t* hq = static_cast<const uint8_t*>(q);
+  const uint8_t* hk = static_cast<const uint8_t*>(k);
+  const uint8_t* hv = static_cast<const uint8_t*>(v);
+  uint8_t* ho = static_cast<uint8_t*>(o);
+  uint8_t* dq = static_cast<uint8_t*>(dev->stage[0]);
+  uint8_t* dk = static_cast<uint8_t*>(dev->stage[1]);
+  uint8_t* dv = static_cast<uint8_t*>(dev->stage[2]);
+  uint8_t* dout = static_cast<uint8_t*>(dev->stage[3]);
+  float* dlse = static_cast<float*>(dev->stage[4]);
+  const size_t q_row = static_cast<size_t>(Hq) * D * 2, kv_row = static_cast<size_t>(Hkv) * D * 2;
+  attn_status_t st = ATTN_OK;
+  for (int b = 0; b < B && ok && st == ATTN_OK; ++b) {
+    int keys_up = 0;  // keys of this batch entry already queued for upload
+    for (int r0 = 0; r0 < Sq && ok && st == ATTN_OK; r0 += chunk_rows) {
+      const int r1 = r0 + chunk_rows < Sq ? r0 + chunk_rows : Sq;
+      const int keys = causal ? (r1 + off < Sk ? r1 + off : Sk) : Sk;  // keys the rows below r1 can see
+      if (keys > keys_up) {
+        const size_t at = (static_cast<size_t>(b) * Sk + keys_up) * kv_row, n = (keys - keys_up) * kv_row;
+        ok = ok && cudaMemcpyAsync(dk + at, hk + at, n, cudaMemcpyHostToDevice, s_up) == cudaSuccess &&
+             cudaMemcpyAsync(dv + at, hv + at, n, cudaMemcpyHostToDevice, s_up) == cudaSuccess;
+        keys_up = keys;
+      }
+      const size_t q_at = (static_cast<size_t>(b) * Sq + r0) * q_row, q_n = static_cast<size_t>(r1 - r0) * q_row;
+      ok = ok && cudaMemcpyAsync(dq + q_at, hq + q_at, q_n, cudaMemcpyHostToDevice, s_up) == cudaSuccess;
+      after(s_run, s_up);
+      if (!ok) break;
+      float* lse_blk = dlse + static_cast<size_t>(b) * Hq * Sq + static_cast<size_t>(Hq) * r0;  // [Hq][r1 - r0]
+      st = fwd_device(dq + q_at, dk + static_cast<size_t>(b) * Sk * kv_row, dv + static_cast<size_t>(b) * Sk * kv_row,
+                      dout + q_at, lse != nullptr ? lse_blk : nullptr, 1, Hq, Hkv, r1 - r0, keys, D,
+                      contiguous_strides(Sq, Hq), contiguous_strides(Sk, Hkv), contiguous_strides(Sk, Hkv),
+                      contiguous_strides(Sq, Hq), causal, scale, s_run);
+      if (st != ATTN_OK) break;
+      after(s_down, s_run);
+      ok = ok && cudaMemcpyAsync(ho + q_at, dout + q_at, q_n, cudaMemcpyDeviceToHost, s_down) == cudaSuccess;
+      if (lse != nullptr) {
+        ok = ok && cudaMemcpy2DAsync(lse + static_cast<size_t>(b) * Hq * Sq + r0, static_cast<size_t>(Sq) * 4, lse_blk,
+                                     static_cast<size_t>(r1 - r0) * 4, static_cast<size_t>(r1 - r0) * 4, Hq,
+                                     cudaMemcpyDeviceToHost, s_down) == cudaSuccess;
+      }
+    }
+  }
+  // join: the caller's stream continues after all three, then the call synchronises it
+  after(user, s_up);
+  after(user, s_run);
+  after(user, s_down);
+  const bool synced = cudaStreamSynchronize(user) == cudaSuccess;
+  if (st != ATTN_OK) return st;
+  return (ok && synced) ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
 }  // namespace
 
 extern "C" {
@@ -346,6 +440,8 @@ attn_status_t attn_fwd_host(const void* q, const void* k, const void* v, void* o
     }
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (g_opt_host_pipeline.load() != 0 && !(causal && Sq > Sk))
+    return host_pipeline(dev, q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, causal, scale, s);
   if (cudaMemcpyAsync(dev->stage[0], q, q_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
       cudaMemcpyAsync(dev->stage[1], k, kv_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
       cudaMemcpyAsync(dev->stage[2], v, kv_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
@@ -453,6 +549,12 @@ attn_status_t attn_release_host_staging(void) {
     d.stage[i] = nullptr;
     d.stage_bytes[i] = 0;
   }
+  for (cudaEvent_t e : d.events) cudaEventDestroy(e);
+  d.events.clear();
+  for (int i = 0; i < 3; ++i) {
+    if (d.pipe[i] != nullptr) cudaStreamDestroy(d.pipe[i]);
+    d.pipe[i] = nullptr;
+  }
   return ATTN_OK;
 }
 
@@ -481,6 +583,11 @@ attn_status_t attn_set_option(const char* name, int value) {
   if (std::strcmp(name, "overlap_epilogue") == 0) {
     if (value < 0 || value > 1) return ATTN_ERR_UNSUPPORTED;
     g_opt_overlap_epilogue.store(value);
+    return ATTN_OK;
+  }
+  if (std::strcmp(name, "host_pipeline") == 0) {
+    if (value < 0 || value > 1) return ATTN_ERR_UNSUPPORTED;
+    g_opt_host_pipeline.store(value);
     return ATTN_OK;
   }
   if (std::strcmp(name, "max_ctas") == 0) {

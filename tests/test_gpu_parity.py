@@ -231,6 +231,31 @@ def test_host_entry_point_matches_device_entry_point():
     lib.attn_release_host_staging()
 
 
+@pytest.mark.parametrize("causal,Sq,Sk", [(False, 2500, 2500), (True, 2500, 2500), (True, 2300, 3000)])
+@pytest.mark.parametrize("pipeline", [1, 0])
+def test_host_entry_point_in_several_chunks(pipeline, causal, Sq, Sk):
+    """32 query heads make a chunk of the pipelined host path 1024 rows, so these problems take
+    three chunks per batch entry (the last one ragged); the result must not depend on the
+    chunking, nor on whether host memory is pinned."""
+    B, Hq, Hkv = 2, 32, 8
+    q, k, v = make_qkv(B, Hq, Hkv, Sq, Sk, 128, seed=7750)
+    o_dev, lse_dev = run_gpu(q, k, v, causal, SCALE)
+    lib.attn_set_option("host_pipeline", pipeline)
+    try:
+        qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+        o = torch.full_like(q, float("nan")).pin_memory()
+        lse = torch.full((B, Hq, Sq), float("nan"), dtype=torch.float32).pin_memory()
+        lib.attn_fwd_host(qh, kh, vh, o, lse, causal, SCALE)
+        assert torch.equal(o.view(torch.int16), o_dev.view(torch.int16))
+        assert torch.equal(lse, lse_dev)
+        o2 = torch.full_like(q, float("nan"))  # pageable, no LSE
+        lib.attn_fwd_host(q, k, v, o2, None, causal, SCALE)
+        assert torch.equal(o2.view(torch.int16), o_dev.view(torch.int16))
+    finally:
+        lib.attn_set_option("host_pipeline", 1)
+        lib.attn_release_host_staging()
+
+
 def test_expired_wait_is_reported_and_the_device_stays_usable():
     """A wait that nothing satisfies runs into its time limit: the kernel returns, the status
     word names the waiter, and the next launches work."""
