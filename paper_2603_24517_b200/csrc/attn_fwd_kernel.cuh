@@ -52,8 +52,9 @@ constexpr int kSmemStage = kSmemKv + kKvSlots * kTileBytes;  // O staging tile f
 constexpr int kSmemStats = kSmemStage + kTileBytes;          // float [2 stages][2][128]
 constexpr int kSmemBars = kSmemStats + 2 * 2 * kTile * 4;
 constexpr int kNumBars = 2 + 2 + 2 * kKvSlots + 2 * 10 + 1;
-constexpr int kSmemMisc = kSmemBars + kNumBars * 8;  // tmem base, abort flag, sched slots
-constexpr int kSmemBytes = kSmemMisc + 32;
+constexpr int kSmemMisc = kSmemBars + kNumBars * 8;  // tmem base, abort flag, two work-item mailbox slots
+constexpr int kMailboxInts = 12;                     // work index + the decoded Work (10 ints), padded
+constexpr int kSmemBytes = kSmemMisc + 8 + 2 * kMailboxInts * 4;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every in-kernel wait gives up after 2 s
@@ -220,18 +221,35 @@ struct Barriers {
 };
 constexpr int kSchedConsumers = 1 + 8 + 4;  // MMA lane, 8 softmax warps, 4 epilogue warps
 
-// Work item of iteration `it` of this CTA for a consumer role (warp-uniform result; < 0 on
-// an expired wait).  `lane_arrives` is true for the one lane per warp that signals consumption.
+// Mailbox slot layout: [0] work index, [1..10] the decoded Work.  The loader decodes an item once,
+// off everybody's critical path (the index arithmetic is a dozen integer divisions), and the other
+// roles copy the result.
+__device__ __forceinline__ void mailbox_put(volatile int* slot, int w, const Work& wk) {
+  slot[1] = wk.b; slot[2] = wk.hkv; slot[3] = wk.hq[0]; slot[4] = wk.hq[1]; slot[5] = wk.row0[0];
+  slot[6] = wk.row0[1]; slot[7] = wk.n[0]; slot[8] = wk.n[1]; slot[9] = wk.nmax;
+  slot[0] = w;
+}
+// Plain loads: the caller has just passed the slot's mbarrier wait (acquire, and a compiler
+// barrier) and signals consumption afterwards, so fields a role never uses cost nothing.
+__device__ __forceinline__ void mailbox_get(const volatile int* vslot, Work& wk) {
+  const int* slot = const_cast<const int*>(vslot);
+  wk.b = slot[1]; wk.hkv = slot[2]; wk.hq[0] = slot[3]; wk.hq[1] = slot[4]; wk.row0[0] = slot[5];
+  wk.row0[1] = slot[6]; wk.n[0] = slot[7]; wk.n[1] = slot[8]; wk.nmax = slot[9];
+}
+
+// Work item of iteration `it` of this CTA for a consumer role: returns its index (warp-uniform;
+// < 0 on an expired wait, >= n_work when the work is exhausted) and fills `wk` for a valid index.
+// `lane_arrives` is true for the one lane per warp that signals consumption.
 __device__ __forceinline__ int consumer_next_work(const FwdParams& p, const Barriers& bars,
                                                   const volatile int* sched_w, int it, WaitCtx ctx, int role,
-                                                  bool lane_arrives, bool whole_warp) {
-  if (!p.dynamic) return static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
-  if (it == 0) return static_cast<int>(blockIdx.x);
-  const int slot = (it - 1) & 1;
-  bool ok = mbar_wait(&bars.sched_full[slot], ((it - 1) >> 1) & 1, ctx, role | kBarSchedFull);
+                                                  bool lane_arrives, bool whole_warp, Work& wk) {
+  const int slot = it & 1;
+  bool ok = mbar_wait(&bars.sched_full[slot], (it >> 1) & 1, ctx, role | kBarSchedFull);
   if (whole_warp) ok = __all_sync(0xffffffffu, ok);
   if (!ok) return -1;
-  const int w = sched_w[slot];
+  const volatile int* box = sched_w + slot * kMailboxInts;
+  const int w = box[0];
+  if (w < p.n_work) mailbox_get(box, wk);
   if (whole_warp) __syncwarp();
   if (lane_arrives) mbar_arrive(&bars.sched_empty[slot]);
   return w;
@@ -290,20 +308,26 @@ __device__ __forceinline__ void role_loader(const FwdParams& p, const Barriers& 
   uint32_t kv_cnt = 0;
   uint32_t q_cnt[2] = {0, 0};
   int w = static_cast<int>(blockIdx.x);
+  Work wk, wk_next;
+  if (w < p.n_work) decode_work(p, w, wk);
+  wk_next = wk;
+  mailbox_put(sched_w, w, wk);  // publication 0 (this CTA's first item) goes to slot 0, which nobody has used yet
+  mbar_arrive(&bars.sched_full[0]);
   for (int it = 0; w < p.n_work; ++it) {
-    // fetch the next work item one item ahead and publish it to the other roles
+    // take the next work item one item ahead, decode it and publish it (publication it + 1)
     int w_next;
     if (p.dynamic) {
-      const int slot = it & 1;
-      if (!mbar_wait(&bars.sched_empty[slot], ((it >> 1) & 1) ^ 1, ctx, kRoleLoad | kBarSchedEmpty)) return;
       w_next = static_cast<int>(atomicAdd(p.counter, 1u)) + static_cast<int>(gridDim.x);
-      sched_w[slot] = w_next;
-      mbar_arrive(&bars.sched_full[slot]);
     } else {
       w_next = w + static_cast<int>(gridDim.x);
     }
-    Work wk;
-    decode_work(p, w, wk);
+    if (w_next < p.n_work) decode_work(p, w_next, wk_next);
+    {
+      const int k = it + 1, slot = k & 1;
+      if (!mbar_wait(&bars.sched_empty[slot], ((k >> 1) & 1) ^ 1, ctx, kRoleLoad | kBarSchedEmpty)) return;
+      mailbox_put(sched_w + slot * kMailboxInts, w_next, wk_next);
+      mbar_arrive(&bars.sched_full[slot]);
+    }
     int q_pending = 0;  // Q tiles are requested after the first K tile so that K never waits behind them
 #pragma unroll
     for (int s = 0; s < 2; ++s) {
@@ -336,6 +360,7 @@ __device__ __forceinline__ void role_loader(const FwdParams& p, const Barriers& 
       }
     }
     w = w_next;
+    wk = wk_next;
   }
 }
 
@@ -354,10 +379,9 @@ __device__ __forceinline__ void role_mma(const FwdParams& p, const Barriers& bar
   uint32_t q_cnt[2] = {0, 0};   // per-stage work items seen (phase of q_full / o_empty)
   uint32_t sp_cnt[2] = {0, 0};  // per-stage K/V blocks seen (phase of p_full)
   for (int it = 0;; ++it) {
-    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleMma, lane == 0, true);
-    if (w < 0 || w >= p.n_work) return;
     Work wk;
-    decode_work(p, w, wk);
+    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleMma, lane == 0, true, wk);
+    if (w < 0 || w >= p.n_work) return;
     // S_s(0) for both stages
     {
       const uint32_t slot = kv_cnt % kKvSlots, par = (kv_cnt / kKvSlots) & 1;
@@ -446,10 +470,9 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
   uint32_t s_cnt = 0;  // phase of s_full[s]
   uint32_t l_cnt = 0;  // phase of l_empty / l_full
   for (int it = 0;; ++it) {
-    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleSoftmax, lane == 0, true);
-    if (w < 0 || w >= p.n_work) return;
     Work wk;
-    decode_work(p, w, wk);
+    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleSoftmax, lane == 0, true, wk);
+    if (w < 0 || w >= p.n_work) return;
     const int n = wk.n[s];
     if (n == 0) continue;
     const int row = wk.row0[s] + row_in_tile;  // global query row (may be >= Sq in a ragged tile)
@@ -575,11 +598,12 @@ __device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers
   uint32_t cnt[2] = {0, 0};
   uint32_t stg_cnt = 0;  // uses of the staging tile so far (phase of stg_empty)
   for (int it = 0;; ++it) {
-    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleEpilogue, lane == 0, true);
-    if (w < 0 || w >= p.n_work) return;
     Work wk;
-    decode_work(p, w, wk);
-#pragma unroll
+    const int w = consumer_next_work(p, bars, sched_w, it, ctx, kRoleEpilogue, lane == 0, true, wk);
+    if (w < 0 || w >= p.n_work) return;
+    // one copy of the code for both stages: a second (unrolled) copy costs registers this role
+    // does not have; the few per-stage values are then indexed at run time
+#pragma unroll 1
     for (int s = 0; s < 2; ++s) {
       if (wk.n[s] == 0) continue;
       const float* stats = reinterpret_cast<const float*>(smem + kSmemStats) + s * 2 * kTile;
