@@ -61,7 +61,10 @@ typedef enum {
  *
  * o must not alias q, k or v.  Distinct streams may call concurrently.  The first
  * call on a device allocates a few KB of library-owned device state (tile-scheduler
- * counters and a status word); tensors are never allocated.
+ * counters and a status word); tensors are never allocated.  After that first call,
+ * attn_fwd issues only a 4-byte cudaMemsetAsync and one kernel launch on `stream`, so it
+ * can be captured into a CUDA graph; replays of one captured call share a work counter
+ * and must not overlap each other.
  * Arithmetic: S and O accumulate in fp32 on the tensor cores; P = exp2 of the scaled,
  * max-subtracted scores is rounded to BF16 before P V; the row sum is taken in fp32
  * before that rounding.

@@ -324,3 +324,36 @@ def test_tiny_workload_in_full():
     q, k, v = make_workload_inputs(w)
     o, lse = run_gpu(q, k, v, w.causal, w.scale)
     check_full(q, k, v, w.causal, w.scale, o, lse)
+
+
+def test_two_streams_and_graph_replay():
+    """Calls on distinct streams may be queued concurrently (each launch takes its own scheduler
+    counter), and a captured call can be replayed: the work counter is reset by a node of the
+    graph itself."""
+    qa, ka, va = make_qkv(1, 4, 4, 700, 700, 128, seed=7900)
+    qb, kb, vb = make_qkv(2, 8, 2, 260, 900, 128, seed=7901)
+    oa_ref, la_ref = run_gpu(qa, ka, va, True, SCALE)
+    ob_ref, lb_ref = run_gpu(qb, kb, vb, False, SCALE)
+    dev = [t.cuda() for t in (qa, ka, va, qb, kb, vb)]
+    oa, ob = torch.empty_like(dev[0]), torch.empty_like(dev[3])
+    la = torch.empty((1, 4, 700), device="cuda", dtype=torch.float32)
+    lb = torch.empty((2, 8, 260), device="cuda", dtype=torch.float32)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        lib.attn_fwd(dev[0], dev[1], dev[2], oa, la, True, SCALE, stream=s1.cuda_stream)
+        lib.attn_fwd(dev[3], dev[4], dev[5], ob, lb, False, SCALE, stream=s2.cuda_stream)
+    torch.cuda.synchronize()
+    assert torch.equal(oa.cpu().view(torch.int16), oa_ref.view(torch.int16)) and torch.equal(la.cpu(), la_ref)
+    assert torch.equal(ob.cpu().view(torch.int16), ob_ref.view(torch.int16)) and torch.equal(lb.cpu(), lb_ref)
+
+    graph = torch.cuda.CUDAGraph()
+    oa.fill_(float("nan"))
+    with torch.cuda.graph(graph):
+        lib.attn_fwd(dev[0], dev[1], dev[2], oa, la, True, SCALE)
+    for _ in range(2):
+        oa.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(oa.cpu().view(torch.int16), oa_ref.view(torch.int16))
+    assert lib.attn_last_device_status()[:2] == (0, 0)
