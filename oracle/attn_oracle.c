@@ -220,3 +220,39 @@ int attn_oracle_merge(const uint16_t *o1, const float *lse1, const uint16_t *o2,
     }
     return 0;
 }
+
+/*
+ * Merge of n partial attention results over pairwise disjoint key sets: the same identity
+ * applied to n parts at once.  LSE = log(sum_i exp(LSE_i)),  O = sum_i exp(LSE_i - LSE) O_i.
+ * o_parts: BF16 bit patterns [n, rows, D]; lse_parts: fp32 [n, rows]; o: double [rows, D];
+ * lse: double [rows].  Parts with LSE = -inf have weight 0; if every part is empty the row is
+ * O = 0, LSE = -inf.
+ */
+int attn_oracle_merge_n(const uint16_t *o_parts, const float *lse_parts, int64_t n, int64_t rows, int64_t D,
+                        double *o, double *lse)
+{
+    if (n <= 0 || rows <= 0 || D <= 0) return 1;
+    for (int64_t r = 0; r < rows; ++r) {
+        double m = -INFINITY;
+        for (int64_t i = 0; i < n; ++i) {
+            const double a = (double)lse_parts[i * rows + r];
+            if (a > m) m = a;
+        }
+        for (int64_t d = 0; d < D; ++d) o[r * D + d] = 0.0;
+        if (m == -INFINITY) {
+            lse[r] = -INFINITY;
+            continue;
+        }
+        double sum = 0.0;
+        for (int64_t i = 0; i < n; ++i) sum += exp((double)lse_parts[i * rows + r] - m);
+        const double tot = m + log(sum);
+        lse[r] = tot;
+        for (int64_t i = 0; i < n; ++i) {
+            const double w = exp((double)lse_parts[i * rows + r] - tot);
+            if (w == 0.0) continue;
+            for (int64_t d = 0; d < D; ++d)
+                o[r * D + d] += w * bf16_to_double(o_parts[(i * rows + r) * D + d]);
+        }
+    }
+    return 0;
+}

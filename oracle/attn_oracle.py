@@ -58,6 +58,8 @@ def _load():
             f32p = ctypes.POINTER(ctypes.c_float)
             lib.attn_oracle_merge.argtypes = [u16p, f32p, u16p, f32p, i64, i64, f64p, f64p]
             lib.attn_oracle_merge.restype = ctypes.c_int
+            lib.attn_oracle_merge_n.argtypes = [u16p, f32p, i64, i64, i64, f64p, f64p]
+            lib.attn_oracle_merge_n.restype = ctypes.c_int
             _lib = lib
     return _lib
 
@@ -146,4 +148,23 @@ def merge(o1, lse1, o2, lse2):
                                    _p(lse, ctypes.c_double))
     if rc != 0:
         raise ValueError(f"attn_oracle_merge failed with code {rc}")
+    return o, lse
+
+
+def merge_n(o_parts, lse_parts):
+    """LSE-weighted merge of n partial results over pairwise disjoint key sets.
+    o_parts: uint16 BF16 bits [n, ..., D]; lse_parts: float32 [n, ...] with one entry per row of a
+    part (same row order).  Returns (O float64 [..., D], LSE float64 [...])."""
+    o_parts = np.ascontiguousarray(o_parts, dtype=np.uint16)
+    lse_parts = np.ascontiguousarray(lse_parts, dtype=np.float32)
+    n, D = o_parts.shape[0], o_parts.shape[-1]
+    rows = o_parts[0].size // D
+    if lse_parts.shape[0] != n or lse_parts[0].size != rows:
+        raise ValueError("inconsistent shapes")
+    o = np.empty(o_parts.shape[1:], dtype=np.float64)
+    lse = np.empty(lse_parts.shape[1:], dtype=np.float64)
+    rc = _load().attn_oracle_merge_n(_p(o_parts, ctypes.c_uint16), _p(lse_parts, ctypes.c_float), n, rows, D,
+                                     _p(o, ctypes.c_double), _p(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"attn_oracle_merge_n failed with code {rc}")
     return o, lse

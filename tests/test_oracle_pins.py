@@ -300,3 +300,81 @@ def test_merge_special_cases():
     # both empty
     o, lse = orc.merge(o1, np.full(5, -np.inf, np.float32), o2, np.full(5, -np.inf, np.float32))
     assert np.all(o == 0) and np.all(lse == -np.inf)
+
+
+def test_merge_n_of_single_key_parts_is_the_softmax_itself():
+    """Pins attn_oracle_merge_n against the definition: n parts of one key each have O_i = v_i and
+    LSE_i = s_i exactly, so their merge is the softmax-weighted mean of the v_i (closed form
+    evaluated here with math.exp)."""
+    vs = [np.array([1.0, -2.0]), np.array([0.5, 4.0]), np.array([-3.0, 0.25]), np.array([8.0, 1.0])]
+    ss = [1.25, -0.75, 0.5, 2.0]  # exactly representable in fp32
+    o, lse = orc.merge_n(np.stack([to_bits(v.reshape(1, 2)) for v in vs]),
+                         np.array([[s] for s in ss], np.float32))
+    z = sum(math.exp(s) for s in ss)
+    want = sum(math.exp(s) / z * v for s, v in zip(ss, vs))
+    np.testing.assert_allclose(o[0], want, atol=1e-14)
+    assert lse[0] == pytest.approx(math.log(z), abs=1e-14)
+
+
+def test_merge_n_special_cases_and_consistency_with_pairwise_merge():
+    parts = np.stack([rand_bits((6, 8), 300 + i) for i in range(4)])
+    lses = np.stack([np.linspace(-2, 2, 6), np.linspace(3, -3, 6), np.full(6, 0.5), np.linspace(0, 1, 6)]).astype(np.float32)
+    o, lse = orc.merge_n(parts, lses)
+    # weights are a probability vector: merging n copies of the same part returns it, LSE + log n
+    same_o, same_l = orc.merge_n(np.stack([parts[0]] * 3), np.stack([lses[0]] * 3))
+    np.testing.assert_allclose(same_o, bits_to_float64(parts[0]), atol=1e-15)
+    np.testing.assert_allclose(same_l, lses[0].astype(np.float64) + math.log(3.0), atol=1e-15)
+    # order of the parts does not matter
+    perm = [2, 0, 3, 1]
+    o_p, lse_p = orc.merge_n(parts[perm], lses[perm])
+    np.testing.assert_allclose(o_p, o, atol=1e-14)
+    np.testing.assert_allclose(lse_p, lse, atol=1e-14)
+    # empty parts (LSE = -inf) have no say; all empty gives O = 0, LSE = -inf
+    lses_e = lses.copy()
+    lses_e[1] = -np.inf
+    o_e, lse_e = orc.merge_n(parts, lses_e)
+    o_3, lse_3 = orc.merge_n(parts[[0, 2, 3]], lses[[0, 2, 3]])
+    np.testing.assert_allclose(o_e, o_3, atol=1e-15)
+    np.testing.assert_allclose(lse_e, lse_3, atol=1e-15)
+    o_0, lse_0 = orc.merge_n(parts, np.full_like(lses, -np.inf))
+    assert np.all(o_0 == 0) and np.all(lse_0 == -np.inf)
+    # n = 2 is the two-part merge
+    o_2, lse_2 = orc.merge_n(parts[:2], lses[:2])
+    o_pair, lse_pair = orc.merge(parts[0], lses[0], parts[1], lses[1])
+    np.testing.assert_allclose(o_2, o_pair, atol=1e-15)
+    np.testing.assert_allclose(lse_2, lse_pair, atol=1e-15)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_split_keys_n_ways_and_merge_equals_the_whole(causal):
+    """The route attn_fwd_splitkv takes, in the oracle alone: attention over key ranges (under the
+    causal mask each range with the offset that keeps global key indices), merged n ways, equals
+    attention over all keys.  The parts are kept in float64 here, so the identity is exact."""
+    B, Hq, Hkv, Sq, Sk, D = 1, 2, 1, 5, 23, 8
+    q, k, v = (bf16_bits(t) for t in make_qkv(B, Hq, Hkv, Sq, Sk, D, seed=310))
+    o, l = orc.attention_full(q, k, v, causal, 0.3)
+    cuts = [0, 6, 7, 16, 23]
+    num = np.zeros_like(o)
+    parts_l = []
+    parts_o = []
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        if causal:
+            # rows see keys j <= i + Sk - Sq; inside the range that is j - lo <= i + (Sk - Sq - lo):
+            # emulate the shifted mask by giving the sub-problem only the keys each row may see
+            o_p = np.zeros_like(o)
+            l_p = np.full(l.shape, -np.inf)
+            for i in range(Sq):
+                last = min(hi, i + Sk - Sq + 1)
+                if last > lo:
+                    oi, li = orc.attention_full(q[:, i:i + 1], k[:, lo:last], v[:, lo:last], False, 0.3)
+                    o_p[:, i] = oi[:, 0]
+                    l_p[:, :, i] = li[:, :, 0]
+        else:
+            o_p, l_p = orc.attention_full(q, k[:, lo:hi], v[:, lo:hi], False, 0.3)
+        parts_o.append(o_p)
+        parts_l.append(l_p)
+    tot = np.log(sum(np.exp(lp) for lp in parts_l))
+    np.testing.assert_allclose(tot, l, atol=1e-13)
+    for o_p, l_p in zip(parts_o, parts_l):
+        num += np.exp(l_p - tot).transpose(0, 2, 1)[..., None] * o_p
+    np.testing.assert_allclose(num, o, atol=1e-13)
