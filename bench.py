@@ -50,9 +50,11 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--op", default="fwd", choices=["fwd", "merge"],
+    ap.add_argument("--op", default="fwd", choices=["fwd", "merge", "splitkv"],
                     help="fwd: the attention forward (default, the headline metric); merge: the LSE-weighted "
-                         "merge of two partial results of the same shape (HBM-bound side kernel)")
+                         "merge of two partial results of the same shape (HBM-bound side kernel); splitkv: "
+                         "one query row per sequence against a long key sequence (decoding shape), attn_fwd "
+                         "against attn_fwd_splitkv for several numbers of key ranges (HBM-bound)")
     ap.add_argument("--sweep", action="store_true",
                     help="time every sequence-length sweep workload (10 warm-ups, then 10 repetitions of 30 launches: "
                          "mean and standard deviation) and print one JSON line with the per-workload TFLOP/s vector "
@@ -414,6 +416,59 @@ def run_sweep(args):
     }), flush=True)
 
 
+def run_splitkv(args):
+    """Decoding shape: B = 4 sequences, 32 query heads on 8 KV heads, ONE query row each, 32768 keys.
+    The K/V tensors (537 MB) must be read once: the path is HBM-bound, and a single launch has only
+    64 work items for 148 SMs.  Times attn_fwd and attn_fwd_splitkv; GB/s = K and V bytes / time."""
+    import paper_2603_24517_b200 as lib
+    from paper_2603_24517_b200 import build as lib_build
+    lib_build.build()
+    lib.load_library()
+    dev = torch.device("cuda", 0)
+    B, Hq, Hkv, Sq, Sk, D = 4, 32, 8, 1, 32768, 128
+    g = torch.Generator(device=dev)
+    g.manual_seed(4242)
+    q = torch.randn((B, Sq, Hq, D), device=dev, generator=g).to(torch.bfloat16)
+    k = torch.randn((B, Sk, Hkv, D), device=dev, generator=g).to(torch.bfloat16)
+    v = torch.randn((B, Sk, Hkv, D), device=dev, generator=g).to(torch.bfloat16)
+    o = torch.empty_like(q)
+    lse = torch.empty((B, Hq, Sq), dtype=torch.float32, device=dev)
+    scale = 1.0 / 128 ** 0.5
+    kv_bytes = 2 * k.numel() * 2
+    results = {}
+    for n in (1, 2, 4, 8, 16, 32):
+        ws = torch.empty(max(16, lib.attn_splitkv_workspace_bytes(B, Hq, Sq, D, n)), dtype=torch.uint8, device=dev)
+        for _ in range(max(3, args.warmup)):
+            lib.attn_fwd_splitkv(q, k, v, o, lse, False, scale, n, workspace=ws)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            lib.attn_fwd_splitkv(q, k, v, o, lse, False, scale, n, workspace=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        results[n] = {"ms": ms, "gbs": kv_bytes / (ms * 1e-3) / 1e9}
+    best = max(results, key=lambda n: results[n]["gbs"])
+    peak, kind = 6650.0, "fallback"
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            peak = float(json.load(f)["hbm_gbs"])
+        kind = "measured"
+    print(json.dumps({
+        "metric": "attn_decode_kv_gbs", "value": results[best]["gbs"], "unit": "GB/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": results[best]["ms"],
+        "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"decode B={B} Hq={Hq} Hkv={Hkv} Sq={Sq} Sk={Sk} D={D} non-causal", "best_n_splits": best,
+                   "l2": f"K and V ({kv_bytes / 2**20:.0f} MiB) exceed the 126 MB L2; no flush"},
+        "by_n_splits": results,
+        "roofline": {"bound": "hbm", "achieved": results[best]["gbs"], "peak": peak, "unit": "GB/s",
+                     "frac": results[best]["gbs"] / peak, "peak_kind": f"{kind} copy bandwidth", "traffic": None,
+                     "algorithmic_bytes": kv_bytes},
+    }), flush=True)
+
+
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of attn_fwd_kernel from the ncu capture
 # summarised in profiles/attn_fwd_kernel_mha_noncausal_s16384_launches.md (402.8 MB + 116.9 MB).
 TRAFFIC_BYTES: dict[str, float | None] = {"mha_noncausal_s16384": 519.7e6}
@@ -428,7 +483,9 @@ def main():
     if args.workload not in workloads:
         raise SystemExit(f"unknown workload {args.workload}; choose from {sorted(workloads)}")
     w = workloads[args.workload]
-    if args.op == "merge":
+    if args.op == "splitkv":
+        run_splitkv(args)
+    elif args.op == "merge":
         run_merge(args, w)
     elif args.impl == "reference":
         run_reference(args, w)

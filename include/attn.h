@@ -33,7 +33,8 @@ typedef enum {
   ATTN_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed (descriptor, launch, copy) */
   ATTN_ERR_ARCH = 6,        /* the current device is not compute capability 10.x */
   ATTN_ERR_TIMEOUT = 7,     /* a bounded wait inside a kernel expired (see attn_last_device_status) */
-  ATTN_ERR_TOO_LARGE = 8    /* attn_fwd_noalloc only: the problem exceeds ATTN_NOALLOC_MAX_Q_TILES */
+  ATTN_ERR_TOO_LARGE = 8    /* attn_fwd_noalloc: the problem exceeds ATTN_NOALLOC_MAX_Q_TILES;
+                               attn_fwd_splitkv: the workspace is too small */
 } attn_status_t;
 
 /*
@@ -234,6 +235,47 @@ attn_status_t attn_last_device_status(int* code, int* detail);
  */
 attn_status_t attn_merge(const void* o1, const float* lse1, const void* o2, const float* lse2,
                          void* o, float* lse, int B, int Hq, int Sq, int D, void* stream);
+
+/*
+ * attn_merge_n -- the same identity for n parts at once (1 <= n <= 64), stored back to back:
+ *
+ *     LSE = log(sum_i exp(LSE_i)),   O = sum_i exp(LSE_i - LSE) * O_i
+ *
+ *   o_parts    BF16 [n][B, Sq, Hq, D] device pointer (read), 16-byte aligned
+ *   lse_parts  FP32 [n][B, Hq, Sq] (read); -inf marks an empty part, whose O_i is not read
+ *   o          BF16 [B, Sq, Hq, D] (written; must not overlap o_parts)
+ *   lse        FP32 [B, Hq, Sq] (written; may be NULL to skip)
+ * Asynchronous on `stream`; fp32 accumulation, one rounding of O to BF16.  Rows whose parts are
+ * all empty get O = 0, LSE = -inf.  ATTN_ERR_UNSUPPORTED for D != 128 or n > 64.
+ */
+attn_status_t attn_merge_n(const void* o_parts, const float* lse_parts, int n, void* o, float* lse,
+                           int B, int Hq, int Sq, int D, void* stream);
+
+/*
+ * attn_fwd_splitkv -- attn_fwd for few query rows against many keys (decoding, short chunks of a
+ * long context), where one launch has too few 256-row work items to fill the GPU.  The key
+ * sequence is cut into up to n_splits ranges of whole 128-key tiles; each range is one launch
+ * of the forward kernel on views of k and v (under the causal mask with the offset that keeps
+ * the global key indices; a range no key of which a row may see leaves that row empty), the
+ * launches run concurrently on library-owned streams, and attn_merge_n combines the partial
+ * results.  The paper's workloads (Sq = Sk) never need this; it is the use the returned LSE
+ * makes possible.
+ *
+ * Arguments as attn_fwd (contiguous layouts), plus:
+ *   n_splits         1..64; fewer ranges are used when Sk is short (one 128-key tile per range
+ *                    at least); with a single range this is attn_fwd
+ *   workspace        device buffer for the partial results, 16-byte aligned, owned by the caller,
+ *                    at least attn_splitkv_workspace_bytes(B, Hq, Sq, D, n_splits) bytes
+ *                    (n_splits * B * Sq * Hq * (2 * D + 4)); may be NULL when n_splits == 1
+ * Result: the same attention; each partial O is rounded to BF16 before the merge, so O carries
+ * up to two more BF16 roundings than attn_fwd's.  Work on `stream` queued before the call is
+ * waited for, and `stream` continues after the merge.  One call at a time per device (the
+ * library's streams and events are shared).  ATTN_ERR_TOO_LARGE if the workspace is too small.
+ */
+size_t attn_splitkv_workspace_bytes(int B, int Hq, int Sq, int D, int n_splits);
+attn_status_t attn_fwd_splitkv(const void* q, const void* k, const void* v, void* o, float* lse,
+                               int B, int Hq, int Hkv, int Sq, int Sk, int D, int causal, float scale,
+                               int n_splits, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * attn_selftest_wait_timeout -- exercises the bounded waits every kernel of this library uses

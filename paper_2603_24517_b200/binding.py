@@ -20,7 +20,8 @@ STATUS_NAMES = {
     0: "ATTN_OK", 1: "ATTN_ERR_NULL", 2: "ATTN_ERR_SHAPE", 3: "ATTN_ERR_UNSUPPORTED", 4: "ATTN_ERR_ALIGN",
     5: "ATTN_ERR_CUDA", 6: "ATTN_ERR_ARCH", 7: "ATTN_ERR_TIMEOUT", 8: "ATTN_ERR_TOO_LARGE",
 }
-EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_strided", "attn_fwd_host", "attn_fwd_noalloc", "attn_merge", "attn_release_host_staging", "attn_set_option",
+EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_strided", "attn_fwd_host", "attn_fwd_noalloc", "attn_merge", "attn_merge_n",
+                    "attn_fwd_splitkv", "attn_splitkv_workspace_bytes", "attn_release_host_staging", "attn_set_option",
                     "attn_plan", "attn_plan_item", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
                     "attn_last_device_status")
 
@@ -63,6 +64,12 @@ def load_library() -> ctypes.CDLL:
     lib.attn_plan_item.restype = ci
     lib.attn_merge.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
     lib.attn_merge.restype = ci
+    lib.attn_merge_n.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, ci, vp]
+    lib.attn_merge_n.restype = ci
+    lib.attn_splitkv_workspace_bytes.argtypes = [ci] * 5
+    lib.attn_splitkv_workspace_bytes.restype = ctypes.c_size_t
+    lib.attn_fwd_splitkv.argtypes = fwd_args[:13] + [ci, vp, ctypes.c_size_t, vp]
+    lib.attn_fwd_splitkv.restype = ci
     lib.attn_selftest_wait_timeout.argtypes = [ci, vp]
     lib.attn_selftest_wait_timeout.restype = ci
     lib.attn_status_str.argtypes = [ci]
@@ -242,6 +249,56 @@ def attn_merge(o1, lse1, o2, lse2, o, lse, stream=None) -> None:
     st = attn_merge_status(o1, lse1, o2, lse2, o, lse, stream)
     if st != ATTN_OK:
         raise AttnError(st, "attn_merge")
+
+
+def attn_merge_n(o_parts, lse_parts, o, lse, stream=None) -> None:
+    """``attn_merge_n`` of the C ABI: o_parts BF16 [n,B,Sq,Hq,D] and lse_parts FP32 [n,B,Hq,Sq]
+    (contiguous) -> o [B,Sq,Hq,D], lse [B,Hq,Sq] (lse may be None)."""
+    if o_parts.dtype != torch.bfloat16 or o_parts.dim() != 5 or not o_parts.is_contiguous() or not o_parts.is_cuda:
+        raise ValueError("o_parts must be a contiguous bfloat16 cuda tensor [n, B, Sq, Hq, D]")
+    n, B, Sq, Hq, D = o_parts.shape
+    if lse_parts.dtype != torch.float32 or not lse_parts.is_contiguous() or tuple(lse_parts.shape) != (n, B, Hq, Sq):
+        raise ValueError("lse_parts must be a contiguous float32 tensor [n, B, Hq, Sq]")
+    if o.dtype != torch.bfloat16 or not o.is_contiguous() or tuple(o.shape) != (B, Sq, Hq, D):
+        raise ValueError("o must be a contiguous bfloat16 tensor [B, Sq, Hq, D]")
+    if lse is not None and (lse.dtype != torch.float32 or not lse.is_contiguous() or tuple(lse.shape) != (B, Hq, Sq)):
+        raise ValueError("lse must be a contiguous float32 tensor [B, Hq, Sq]")
+    if stream is None:
+        stream = torch.cuda.current_stream(o.device).cuda_stream
+    with torch.cuda.device(o.device):
+        st = load_library().attn_merge_n(o_parts.data_ptr(), lse_parts.data_ptr(), n, o.data_ptr(),
+                                         None if lse is None else lse.data_ptr(), B, Hq, Sq, D, stream)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_merge_n")
+
+
+def attn_splitkv_workspace_bytes(B: int, Hq: int, Sq: int, D: int, n_splits: int) -> int:
+    return int(load_library().attn_splitkv_workspace_bytes(B, Hq, Sq, D, n_splits))
+
+
+def attn_fwd_splitkv_status(q, k, v, o, lse, causal: bool, scale: float, n_splits: int, workspace=None,
+                            stream=None) -> int:
+    """Calls ``attn_fwd_splitkv``; ``workspace`` is a uint8 cuda tensor (allocated here when None)."""
+    B, Hq, Hkv, Sq, Sk, D = _check_layout(q, k, v, o, lse, "cuda")
+    need = attn_splitkv_workspace_bytes(B, Hq, Sq, D, n_splits) if 1 <= n_splits <= 64 else 0
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        return load_library().attn_fwd_splitkv(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                               None if lse is None else lse.data_ptr(), B, Hq, Hkv, Sq, Sk, D,
+                                               int(bool(causal)), float(scale), int(n_splits),
+                                               None if workspace is None else workspace.data_ptr(),
+                                               0 if workspace is None else workspace.numel(), stream)
+
+
+def attn_fwd_splitkv(q, k, v, o, lse, causal: bool, scale: float, n_splits: int, workspace=None, stream=None) -> None:
+    """``attn_fwd_splitkv`` of the C ABI: the forward with the key sequence cut into up to
+    ``n_splits`` ranges that run concurrently and are merged (for few query rows, many keys)."""
+    st = attn_fwd_splitkv_status(q, k, v, o, lse, causal, scale, n_splits, workspace, stream)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_fwd_splitkv")
 
 
 def attn_selftest_wait_timeout(limit_ms: int, device=0, stream=None) -> None:

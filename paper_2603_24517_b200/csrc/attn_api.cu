@@ -21,6 +21,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 constexpr int kMaxDevices = 64;
 constexpr int kCounterSlots = 1024;  // one work counter per launch in flight, reused round-robin
+constexpr int kSplitStreams = 8;
+constexpr int kMaxSplits = 64;
 
 struct DeviceState {
   bool ready = false;
@@ -35,6 +37,8 @@ struct DeviceState {
   // attn_fwd_host pipeline: upload, compute and download streams and a pool of events
   cudaStream_t pipe[3] = {nullptr, nullptr, nullptr};
   std::vector<cudaEvent_t> events;
+  // attn_fwd_splitkv: streams the key ranges are launched on, so that their small grids share the GPU
+  cudaStream_t split[kSplitStreams] = {};
 };
 
 std::mutex g_mutex;
@@ -264,6 +268,11 @@ attn_status_t attn_plan_item(int B, int Hq, int Hkv, int Sq, int Sk, int D, int 
 
 namespace {
 
+// Causal rule used by the kernels: key j of the K/V passed in is visible to query row i iff
+// j <= i + off.  off = Sk - Sq by default (bottom-right alignment); a launch on a key range of a
+// longer sequence passes the offset that keeps the global key indices.
+constexpr long long kDefaultCausalOff = -(1ll << 62);
+
 // A stride the TMA engine accepts: positive, a multiple of 8 elements (16 bytes), below 2^40
 // bytes; axes of extent 1 are never stepped along, but the descriptor still wants a legal value.
 attn_status_t check_strides(const long long* s) {
@@ -279,7 +288,7 @@ attn_status_t check_strides(const long long* s) {
 
 attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
                          int Sq, int Sk, int D, Strides3 sq, Strides3 sk, Strides3 sv, Strides3 so, int causal,
-                         float scale, void* stream) {
+                         float scale, void* stream, long long causal_off = kDefaultCausalOff) {
   attn_status_t st = check_args(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, scale, true);
   if (st != ATTN_OK) return st;
   DeviceState* dev = device_state(&st);
@@ -292,6 +301,7 @@ attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, f
 
   FwdParams p;
   fill_plan(&p, B, Hq, Hkv, Sq, Sk, causal);
+  if (causal_off != kDefaultCausalOff) p.off = static_cast<int>(causal_off);
   p.scale = scale;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.lse = lse;
@@ -555,6 +565,10 @@ attn_status_t attn_release_host_staging(void) {
     if (d.pipe[i] != nullptr) cudaStreamDestroy(d.pipe[i]);
     d.pipe[i] = nullptr;
   }
+  for (int i = 0; i < kSplitStreams; ++i) {
+    if (d.split[i] != nullptr) cudaStreamDestroy(d.split[i]);
+    d.split[i] = nullptr;
+  }
   return ATTN_OK;
 }
 
@@ -621,6 +635,93 @@ attn_status_t attn_merge(const void* o1, const float* lse1, const void* o2, cons
       static_cast<const uint4*>(o1), lse1, static_cast<const uint4*>(o2), lse2, static_cast<uint4*>(o), lse, Hq, Sq,
       n_chunks);
   return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+attn_status_t attn_merge_n(const void* o_parts, const float* lse_parts, int n, void* o, float* lse, int B, int Hq,
+                           int Sq, int D, void* stream) {
+  if (o_parts == nullptr || lse_parts == nullptr || o == nullptr) return ATTN_ERR_NULL;
+  if (B <= 0 || Hq <= 0 || Sq <= 0 || D <= 0 || n <= 0) return ATTN_ERR_SHAPE;
+  if (D != attn::kHeadDim || n > kMaxSplits) return ATTN_ERR_UNSUPPORTED;
+  const uintptr_t mask = 15;
+  if ((reinterpret_cast<uintptr_t>(o_parts) & mask) || (reinterpret_cast<uintptr_t>(o) & mask) ||
+      (reinterpret_cast<uintptr_t>(lse_parts) & 3) || (reinterpret_cast<uintptr_t>(lse) & 3))
+    return ATTN_ERR_ALIGN;
+  attn_status_t st = ATTN_OK;
+  DeviceState* dev = device_state(&st);
+  if (dev == nullptr) return st;
+  const long long n_rows = static_cast<long long>(B) * Sq * Hq;
+  const long long n_chunks = n_rows * attn::kChunksPerRow;
+  long long blocks = (n_chunks + attn::kMergeThreads - 1) / attn::kMergeThreads;
+  const long long cap = static_cast<long long>(dev->sm_count) * 8;
+  if (blocks > cap) blocks = cap;
+  attn::attn_merge_n_kernel<<<static_cast<int>(blocks), attn::kMergeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint4*>(o_parts), lse_parts, n, static_cast<uint4*>(o), lse, Hq, Sq, n_chunks, n_rows);
+  return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+size_t attn_splitkv_workspace_bytes(int B, int Hq, int Sq, int D, int n_splits) {
+  if (B <= 0 || Hq <= 0 || Sq <= 0 || D != attn::kHeadDim || n_splits <= 0 || n_splits > kMaxSplits) return 0;
+  const size_t rows = static_cast<size_t>(B) * Sq * Hq;
+  return static_cast<size_t>(n_splits) * rows * (static_cast<size_t>(D) * 2 + 4);
+}
+
+attn_status_t attn_fwd_splitkv(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq,
+                               int Hkv, int Sq, int Sk, int D, int causal, float scale, int n_splits,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+  attn_status_t st = check_args(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, scale, true);
+  if (st != ATTN_OK) return st;
+  if (n_splits <= 0) return ATTN_ERR_SHAPE;
+  if (n_splits > kMaxSplits) return ATTN_ERR_UNSUPPORTED;
+  // key ranges of whole 128-key tiles, all but the last of equal length
+  const int per = (Sk + n_splits - 1) / n_splits;
+  const int len = (per + attn::kTile - 1) / attn::kTile * attn::kTile;
+  const int n = (Sk + len - 1) / len;
+  const Strides3 sq = contiguous_strides(Sq, Hq), sk = contiguous_strides(Sk, Hkv);
+  if (n == 1) return fwd_device(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, sq, sk, sk, sq, causal, scale, stream);
+  if (workspace == nullptr) return ATTN_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(workspace) & 15) return ATTN_ERR_ALIGN;
+  if (workspace_bytes < attn_splitkv_workspace_bytes(B, Hq, Sq, D, n)) return ATTN_ERR_TOO_LARGE;
+  DeviceState* dev = device_state(&st);
+  if (dev == nullptr) return st;
+  for (int i = 0; i < kSplitStreams && i < n; ++i) {
+    if (dev->split[i] == nullptr &&
+        cudaStreamCreateWithFlags(&dev->split[i], cudaStreamNonBlocking) != cudaSuccess)
+      return ATTN_ERR_CUDA;
+  }
+  const cudaStream_t user = static_cast<cudaStream_t>(stream);
+  size_t next_event = 0;
+  bool ok = true;
+  auto after = [&](cudaStream_t waiter, cudaStream_t signaller) {
+    if (next_event == dev->events.size()) {
+      cudaEvent_t e = nullptr;
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) {
+        ok = false;
+        return;
+      }
+      dev->events.push_back(e);
+    }
+    cudaEvent_t e = dev->events[next_event++];
+    ok = ok && cudaEventRecord(e, signaller) == cudaSuccess && cudaStreamWaitEvent(waiter, e, 0) == cudaSuccess;
+  };
+  const int used = n < kSplitStreams ? n : kSplitStreams;
+  for (int i = 0; i < used; ++i) after(dev->split[i], user);
+  const size_t rows = static_cast<size_t>(B) * Sq * Hq;
+  uint8_t* o_parts = static_cast<uint8_t*>(workspace);
+  float* lse_parts = reinterpret_cast<float*>(o_parts + static_cast<size_t>(n) * rows * D * 2);
+  const uint8_t* kb = static_cast<const uint8_t*>(k);
+  const uint8_t* vb = static_cast<const uint8_t*>(v);
+  for (int i = 0; i < n && ok && st == ATTN_OK; ++i) {
+    const int k0 = i * len, k1 = (k0 + len < Sk) ? k0 + len : Sk;
+    const size_t kv_at = static_cast<size_t>(k0) * Hkv * D * 2;
+    // rows see keys j <= row + (Sk - Sq) of the whole sequence, i.e. j - k0 <= row + (Sk - Sq - k0) of this range
+    st = fwd_device(q, kb + kv_at, vb + kv_at, o_parts + static_cast<size_t>(i) * rows * D * 2,
+                    lse_parts + static_cast<size_t>(i) * rows, B, Hq, Hkv, Sq, k1 - k0, D, sq, sk, sk, sq, causal,
+                    scale, dev->split[i % kSplitStreams], static_cast<long long>(Sk) - Sq - k0);
+  }
+  for (int i = 0; i < used; ++i) after(user, dev->split[i]);
+  if (st != ATTN_OK) return st;
+  if (!ok) return ATTN_ERR_CUDA;
+  return attn_merge_n(o_parts, lse_parts, n, o, lse, B, Hq, Sq, D, stream);
 }
 
 attn_status_t attn_selftest_wait_timeout(int limit_ms, void* stream) {

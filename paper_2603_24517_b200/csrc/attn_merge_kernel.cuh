@@ -73,4 +73,48 @@ attn_merge_kernel(const uint4* __restrict__ o1, const float* __restrict__ lse1, 
   }
 }
 
+// The same merge for n parts stored back to back: o_parts [n][B, Sq, Hq, 128] BF16, lse_parts
+// [n][B, Hq, Sq] fp32.  LSE = log(sum_i exp(LSE_i)), O = sum_i exp(LSE_i - LSE) O_i, accumulated in
+// fp32 and rounded once.  The n LSE values of a row are read by the 16 threads that share the row
+// (same addresses: one transaction each).
+__global__ void __launch_bounds__(kMergeThreads)
+attn_merge_n_kernel(const uint4* __restrict__ o_parts, const float* __restrict__ lse_parts, int n,
+                    uint4* __restrict__ o, float* __restrict__ lse, int Hq, int Sq, long long n_chunks,
+                    long long n_rows) {
+  const long long stride = static_cast<long long>(gridDim.x) * kMergeThreads;
+  for (long long c = static_cast<long long>(blockIdx.x) * kMergeThreads + threadIdx.x; c < n_chunks; c += stride) {
+    const long long row = c / kChunksPerRow;  // (b * Sq + i) * Hq + h
+    const int h = static_cast<int>(row % Hq);
+    const long long t = row / Hq;
+    const int i = static_cast<int>(t % Sq);
+    const long long b = t / Sq;
+    const long long li = (b * Hq + h) * Sq + i;  // LSE is [B, Hq, Sq]
+    float m = -INFINITY;
+    for (int p = 0; p < n; ++p) m = fmaxf(m, __ldg(lse_parts + p * n_rows + li));
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    float tot = -INFINITY;
+    if (m != -INFINITY) {
+      float sum = 0.f;
+      for (int p = 0; p < n; ++p) sum += expf(__ldg(lse_parts + p * n_rows + li) - m);
+      tot = m + logf(sum);
+      for (int p = 0; p < n; ++p) {
+        const float w = expf(__ldg(lse_parts + p * n_rows + li) - tot);
+        if (w == 0.f) continue;  // an empty part may hold anything, also NaN from an untouched buffer
+        const uint4 x = __ldg(o_parts + p * n_chunks + c);
+        acc[0] = fmaf(w, bf16_lo(x.x), acc[0]); acc[1] = fmaf(w, bf16_hi(x.x), acc[1]);
+        acc[2] = fmaf(w, bf16_lo(x.y), acc[2]); acc[3] = fmaf(w, bf16_hi(x.y), acc[3]);
+        acc[4] = fmaf(w, bf16_lo(x.z), acc[4]); acc[5] = fmaf(w, bf16_hi(x.z), acc[5]);
+        acc[6] = fmaf(w, bf16_lo(x.w), acc[6]); acc[7] = fmaf(w, bf16_hi(x.w), acc[7]);
+      }
+    }
+    uint4 r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r.x) : "f"(acc[1]), "f"(acc[0]));
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r.y) : "f"(acc[3]), "f"(acc[2]));
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r.z) : "f"(acc[5]), "f"(acc[4]));
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r.w) : "f"(acc[7]), "f"(acc[6]));
+    o[c] = r;
+    if (lse != nullptr && (c % kChunksPerRow) == 0) lse[li] = tot;
+  }
+}
+
 }  // namespace attn
