@@ -450,6 +450,29 @@ def run_splitkv(args):
         ms = e0.elapsed_time(e1) / args.steps
         results[n] = {"ms": ms, "gbs": kv_bytes / (ms * 1e-3) / 1e9}
     best = max(results, key=lambda n: results[n]["gbs"])
+    # a chunk of a long context: 512 query rows against 65536 keys, 16 heads (tensor-bound, but only
+    # 32 work items in one launch)
+    Bc, Hc, Sqc, Skc = 1, 16, 512, 65536
+    qc = torch.randn((Bc, Sqc, Hc, D), device=dev, generator=g).to(torch.bfloat16)
+    kc = torch.randn((Bc, Skc, Hc, D), device=dev, generator=g).to(torch.bfloat16)
+    vc = torch.randn((Bc, Skc, Hc, D), device=dev, generator=g).to(torch.bfloat16)
+    oc = torch.empty_like(qc)
+    lc = torch.empty((Bc, Hc, Sqc), dtype=torch.float32, device=dev)
+    chunk_flops = 4.0 * Bc * Hc * Sqc * Skc * D
+    chunk = {}
+    for n in (1, 2, 4, 8):
+        ws = torch.empty(max(16, lib.attn_splitkv_workspace_bytes(Bc, Hc, Sqc, D, n)), dtype=torch.uint8, device=dev)
+        for _ in range(max(3, args.warmup)):
+            lib.attn_fwd_splitkv(qc, kc, vc, oc, lc, False, scale, n, workspace=ws)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            lib.attn_fwd_splitkv(qc, kc, vc, oc, lc, False, scale, n, workspace=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        chunk[n] = {"ms": ms, "tflops": chunk_flops / (ms * 1e-3) / 1e12}
     peak, kind = 6650.0, "fallback"
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -463,6 +486,7 @@ def run_splitkv(args):
         "config": {"workload": f"decode B={B} Hq={Hq} Hkv={Hkv} Sq={Sq} Sk={Sk} D={D} non-causal", "best_n_splits": best,
                    "l2": f"K and V ({kv_bytes / 2**20:.0f} MiB) exceed the 126 MB L2; no flush"},
         "by_n_splits": results,
+        "context_chunk": {"workload": f"B={Bc} H={Hc} Sq={Sqc} Sk={Skc} D={D} non-causal", "by_n_splits": chunk},
         "roofline": {"bound": "hbm", "achieved": results[best]["gbs"], "peak": peak, "unit": "GB/s",
                      "frac": results[best]["gbs"] / peak, "peak_kind": f"{kind} copy bandwidth", "traffic": None,
                      "algorithmic_bytes": kv_bytes},
