@@ -170,6 +170,10 @@ attn_status_t attn_release_host_staging(void);
  *   "overlap_epilogue"  1 (default) = a query stage is normalised and stored as soon as its own
  *                 last P V has completed, overlapping the other stage's (Section 5.2);
  *                 0 = only after both stages' last P V ("kernel" = 0 only)
+ *   "gqa_pack"    1 (default) = when a GQA group's query rows all fit two tiles
+ *                 (Sq <= 2 * 128 / group, group a power of two <= 16, "kernel" = 0), the heads of
+ *                 a KV group share the rows of a tile, so its K/V is streamed once for the whole
+ *                 group (decoding, short chunks); results are bit-identical; 0 = never
  *   "host_pipeline"  1 (default) = attn_fwd_host overlaps upload, compute and download in row
  *                 chunks; 0 = one upload, one launch, one download
  *   "kernel"      0 = dual query stage: a CTA runs two 128-row query tiles against one stream

@@ -51,6 +51,7 @@ std::atomic<int> g_opt_rescale_threshold{8};
 std::atomic<int> g_opt_split_p{1};
 std::atomic<int> g_opt_overlap_epilogue{1};
 std::atomic<int> g_opt_host_pipeline{1};
+std::atomic<int> g_opt_gqa_pack{1};
 
 // Per-device one-time set-up: architecture check, kernel attribute, scheduler counters and
 // status word.  Returns the state or nullptr (with *st set).
@@ -113,12 +114,13 @@ Strides3 contiguous_strides(int S, int H) {
 
 // BF16 tensor seen as 4-D (D, H, S, B) with the given element strides; box = 64 elements x 1 head
 // x 128 rows, 128-byte swizzle, out-of-range rows read as zero and are clipped on store.
-bool make_tensor_map(CUtensorMap* tm, const void* base, int B, int S, int H, Strides3 st) {
+bool make_tensor_map(CUtensorMap* tm, const void* base, int B, int S, int H, Strides3 st, int pack_log2 = 0) {
   const cuuint64_t dims[4] = {128, static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(S),
                               static_cast<cuuint64_t>(B)};
   const cuuint64_t strides[3] = {static_cast<cuuint64_t>(st.h) * 2, static_cast<cuuint64_t>(st.s) * 2,
                                  static_cast<cuuint64_t>(st.b) * 2};
-  const cuuint32_t box[4] = {64, 1, 128, 1};
+  // packed query tiles: `group` heads x (128 / group) rows, laid out row-major as (row, head)
+  const cuuint32_t box[4] = {64, 1u << pack_log2, 128u >> pack_log2, 1};
   const cuuint32_t elem_strides[4] = {1, 1, 1, 1};
   return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                   elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -155,7 +157,19 @@ void fill_plan(FwdParams* p, int B, int Hq, int Hkv, int Sq, int Sk, int causal)
   p->n_qt = (Sq + attn::kTile - 1) / attn::kTile;
   p->n_kb = (Sk + attn::kTile - 1) / attn::kTile;
   p->kernel = g_opt_kernel.load();
-  if (p->kernel == 1) {  // triple score buffer: one query tile per work item
+  // Short query sequences of a GQA group (all of it fits two packed tiles): pack the group's
+  // heads into the rows of a tile, so that each KV head is streamed once per row tile pair.
+  p->pack_log2 = 0;
+  if (g_opt_gqa_pack.load() != 0 && p->kernel == 0 && p->group >= 2 && p->group <= 16 &&
+      (p->group & (p->group - 1)) == 0 && Sq <= 2 * (attn::kTile / p->group)) {
+    while ((1 << p->pack_log2) < p->group) ++p->pack_log2;
+  }
+  if (p->pack_log2 > 0) {
+    p->n_qt = (Sq + (attn::kTile >> p->pack_log2) - 1) / (attn::kTile >> p->pack_log2);
+    p->pair_heads = 0;
+    p->items_per_group = (p->n_qt + 1) / 2;
+    p->n_work = B * Hkv * p->items_per_group;
+  } else if (p->kernel == 1) {  // triple score buffer: one query tile per work item
     p->pair_heads = 0;
     p->items_per_group = p->n_qt;
     p->n_work = B * Hq * p->n_qt;
@@ -294,14 +308,15 @@ attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, f
   DeviceState* dev = device_state(&st);
   if (dev == nullptr) return st;
 
-  CUtensorMap tm_q, tm_k, tm_v, tm_o;
-  if (!make_tensor_map(&tm_q, q, B, Sq, Hq, sq) || !make_tensor_map(&tm_k, k, B, Sk, Hkv, sk) ||
-      !make_tensor_map(&tm_v, v, B, Sk, Hkv, sv) || !make_tensor_map(&tm_o, o, B, Sq, Hq, so))
-    return ATTN_ERR_CUDA;
-
   FwdParams p;
   fill_plan(&p, B, Hq, Hkv, Sq, Sk, causal);
   if (causal_off != kDefaultCausalOff) p.off = static_cast<int>(causal_off);
+
+  CUtensorMap tm_q, tm_k, tm_v, tm_o;
+  if (!make_tensor_map(&tm_q, q, B, Sq, Hq, sq, p.pack_log2) || !make_tensor_map(&tm_k, k, B, Sk, Hkv, sk) ||
+      !make_tensor_map(&tm_v, v, B, Sk, Hkv, sv) || !make_tensor_map(&tm_o, o, B, Sq, Hq, so, p.pack_log2))
+    return ATTN_ERR_CUDA;
+
   p.scale = scale;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.lse = lse;
@@ -529,15 +544,16 @@ attn_status_t attn_fwd_noalloc(const void* q, const void* k, const void* v, void
   st = noalloc_device(&dev);
   if (st != ATTN_OK) return st;
 
-  CUtensorMap tm_q, tm_k, tm_v, tm_o;
-  if (!make_tensor_map(&tm_q, q, B, Sq, Hq, contiguous_strides(Sq, Hq)) ||
-      !make_tensor_map(&tm_k, k, B, Sk, Hkv, contiguous_strides(Sk, Hkv)) ||
-      !make_tensor_map(&tm_v, v, B, Sk, Hkv, contiguous_strides(Sk, Hkv)) ||
-      !make_tensor_map(&tm_o, o, B, Sq, Hq, contiguous_strides(Sq, Hq)))
-    return ATTN_ERR_CUDA;
-
   FwdParams p;
   fill_plan(&p, B, Hq, Hkv, Sq, Sk, causal);
+
+  CUtensorMap tm_q, tm_k, tm_v, tm_o;
+  if (!make_tensor_map(&tm_q, q, B, Sq, Hq, contiguous_strides(Sq, Hq), p.pack_log2) ||
+      !make_tensor_map(&tm_k, k, B, Sk, Hkv, contiguous_strides(Sk, Hkv)) ||
+      !make_tensor_map(&tm_v, v, B, Sk, Hkv, contiguous_strides(Sk, Hkv)) ||
+      !make_tensor_map(&tm_o, o, B, Sq, Hq, contiguous_strides(Sq, Hq), p.pack_log2))
+    return ATTN_ERR_CUDA;
+
   p.scale = scale;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.lse = lse;
@@ -597,6 +613,11 @@ attn_status_t attn_set_option(const char* name, int value) {
   if (std::strcmp(name, "overlap_epilogue") == 0) {
     if (value < 0 || value > 1) return ATTN_ERR_UNSUPPORTED;
     g_opt_overlap_epilogue.store(value);
+    return ATTN_OK;
+  }
+  if (std::strcmp(name, "gqa_pack") == 0) {
+    if (value < 0 || value > 1) return ATTN_ERR_UNSUPPORTED;
+    g_opt_gqa_pack.store(value);
     return ATTN_OK;
   }
   if (std::strcmp(name, "host_pipeline") == 0) {

@@ -68,6 +68,10 @@ struct FwdParams {
   int n_kb;         // ceil(Sk / 128)
   int pair_heads;   // 1: the two stages hold two query heads of one KV head at the same rows
                     // 0: the two stages hold two consecutive row tiles of one query head
+  int pack_log2;    // > 0 (short query sequences, "kernel" 0 only): a tile's 128 rows hold
+                    // 128 >> pack_log2 query rows of ALL group = 1 << pack_log2 query heads of one KV
+                    // head (tile row r = query row r / group, head r % group), so a KV head's K/V is
+                    // streamed once for its whole group; the stages hold two consecutive row tiles
   int items_per_group;  // work items per (b, hq) [pair rows] or per (b, hkv) [pair heads]
   int n_work;
   int dynamic;      // 1: work items come from the global counter
@@ -134,18 +138,25 @@ __host__ __device__ __forceinline__ void decode_work(const FwdParams& p, int w, 
     wk.row0[0] = wk.row0[1] = qt * kTile;
   } else {
     int qp = p.causal ? (p.items_per_group - 1 - r) : r;
-    wk.b = grp / p.Hq;
-    wk.hq[0] = wk.hq[1] = grp - wk.b * p.Hq;
-    wk.hkv = wk.hq[0] / p.group;
-    wk.row0[0] = qp * 2 * kTile;
-    wk.row0[1] = wk.row0[0] + kTile;
+    if (p.pack_log2 > 0) {  // groups are (batch, KV head); hq is the first query head of the group
+      wk.b = grp / p.Hkv;
+      wk.hkv = grp - wk.b * p.Hkv;
+      wk.hq[0] = wk.hq[1] = wk.hkv * p.group;
+    } else {
+      wk.b = grp / p.Hq;
+      wk.hq[0] = wk.hq[1] = grp - wk.b * p.Hq;
+      wk.hkv = wk.hq[0] / p.group;
+    }
+    wk.row0[0] = qp * 2 * (kTile >> p.pack_log2);
+    wk.row0[1] = wk.row0[0] + (kTile >> p.pack_log2);
   }
+  const int tile_rows = kTile >> p.pack_log2;  // query rows per tile
 #pragma unroll
   for (int s = 0; s < 2; ++s) {
     if (wk.row0[s] >= p.Sq) {
       wk.n[s] = 0;
     } else if (p.causal) {
-      const int row_end = wk.row0[s] + kTile < p.Sq ? wk.row0[s] + kTile : p.Sq;
+      const int row_end = wk.row0[s] + tile_rows < p.Sq ? wk.row0[s] + tile_rows : p.Sq;
       // a tile none of whose rows sees a key (Sq > Sk) still visits one, fully masked, block, so
       // that its O = 0 and LSE = -inf are produced by the ordinary path
       const int last_key = row_end - 1 + p.off;
@@ -475,7 +486,7 @@ __device__ __forceinline__ void role_softmax(const FwdParams& p, const Barriers&
     if (w < 0 || w >= p.n_work) return;
     const int n = wk.n[s];
     if (n == 0) continue;
-    const int row = wk.row0[s] + row_in_tile;  // global query row (may be >= Sq in a ragged tile)
+    const int row = wk.row0[s] + (row_in_tile >> p.pack_log2);  // global query row (may be >= Sq in a ragged tile)
     // number of keys this row may see, counted from key 0
     const int row_limit = p.causal ? min(p.Sk, row + p.off + 1) : p.Sk;
     // first key index from which a block needs per-element masking for this tile
@@ -652,9 +663,10 @@ __device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers
       }
       tc_fence_before_sync();
       if (lane == 0) mbar_arrive(&bars.o_empty[s]);
-      const int row = wk.row0[s] + row_in_tile;
+      const int row = wk.row0[s] + (row_in_tile >> p.pack_log2);
+      const int head = wk.hq[s] + (row_in_tile & ((1 << p.pack_log2) - 1));
       if (p.lse != nullptr && row < p.Sq) {
-        p.lse[(static_cast<size_t>(wk.b) * p.Hq + wk.hq[s]) * p.Sq + row] = m_used * p.scale + logf(l);
+        p.lse[(static_cast<size_t>(wk.b) * p.Hq + head) * p.Sq + row] = m_used * p.scale + logf(l);
       }
       fence_proxy_async_smem();
       __syncwarp();

@@ -93,3 +93,50 @@ def test_splitkv_argument_errors_and_workspace():
     ws = torch.empty(need, dtype=torch.uint8, device="cuda")
     assert lib.attn_fwd_splitkv_status(q, k, v, o, None, False, SCALE, 4, workspace=ws) == 0       # lse may be NULL
     torch.cuda.synchronize()
+
+
+# ---- short GQA query sequences: the heads of a KV group packed into the rows of one tile --------
+PACKED = [
+    # B, Hq, Hkv, Sq, Sk, causal
+    (2, 8, 2, 1, 700, False),      # decoding, group 4: rows 0..3 of a tile are the 4 heads
+    (2, 8, 2, 1, 700, True),
+    (1, 8, 2, 17, 300, True),      # 17 rows x 4 heads in one tile of 32 x 4
+    (2, 8, 2, 40, 700, True),      # two packed tiles: both stages busy, ragged second tile
+    (1, 8, 2, 64, 64, True),       # Sq = Sk, diagonal inside the packed tiles
+    (1, 8, 1, 32, 515, False),     # group 8: two tiles of 16 rows
+    (1, 8, 1, 5, 130, True),
+    (3, 4, 2, 128, 128, True),     # group 2: two tiles of 64 rows
+    (1, 16, 1, 9, 1000, False),    # group 16: 8 rows per tile
+    (1, 8, 2, 20, 9, True),        # Sq > Sk: packed rows without any visible key
+]
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,causal", PACKED)
+def test_packed_gqa_tiles_match_oracle_and_the_unpacked_path(B, Hq, Hkv, Sq, Sk, causal):
+    plan = lib.attn_plan(B, Hq, Hkv, Sq, Sk, 128, causal, 148)
+    assert plan["n_work"] == B * Hkv * math.ceil(math.ceil(Sq / (128 // (Hq // Hkv))) / 2)   # the packed plan is in use
+    q, k, v = make_qkv(B, Hq, Hkv, Sq, Sk, 128, seed=9800 + Sq)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    outs = []
+    for pack in (1, 0):
+        lib.attn_set_option("gqa_pack", pack)
+        try:
+            o = torch.full_like(qd, float("nan"))
+            lse = torch.full((B, Hq, Sq), float("nan"), device="cuda")
+            lib.attn_fwd(qd, kd, vd, o, lse, causal, SCALE)
+            torch.cuda.synchronize()
+            assert lib.attn_last_device_status()[:2] == (0, 0)
+            outs.append((o.cpu(), lse.cpu()))
+        finally:
+            lib.attn_set_option("gqa_pack", 1)
+    # per row the arithmetic is the same in both layouts
+    assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16))
+    assert torch.equal(outs[0][1], outs[1][1])
+    o_ref, l_ref = orc.attention_full(bf16_bits(q), bf16_bits(k), bf16_bits(v), causal, SCALE)
+    o64 = bits_to_float64(bf16_bits(outs[0][0]))
+    l64 = outs[0][1].numpy().astype(np.float64)
+    assert not np.isnan(o64).any() and not np.isnan(l64).any()
+    assert np.abs(o64 - o_ref).max() <= TOL_O
+    empty = np.isneginf(l_ref)
+    assert np.array_equal(np.isneginf(l64), empty)
+    assert np.abs(l64[~empty] - l_ref[~empty]).max() <= TOL_LSE

@@ -22,8 +22,17 @@ def _built():
     lib.attn_set_option("kernel", 0)
 
 
-def visible_blocks_brute(row0, Sq, Sk, causal):
-    rows = range(row0, min(row0 + TILE, Sq))
+def packed_group(Hq, Hkv, Sq):
+    """Query heads per tile row group when the library packs a GQA group into one tile (short
+    query sequences, dual-stage kernel): the whole group must fit two packed tiles."""
+    g = Hq // Hkv
+    if 2 <= g <= 16 and g & (g - 1) == 0 and Sq <= 2 * (TILE // g):
+        return g
+    return 1
+
+
+def visible_blocks_brute(row0, Sq, Sk, causal, tile_rows=TILE):
+    rows = range(row0, min(row0 + tile_rows, Sq))
     if not causal:
         return math.ceil(Sk / TILE)
     last_key = max(min(Sk - 1, i + Sk - Sq) for i in rows)
@@ -38,6 +47,8 @@ CASES = [
     (1, 32, 4, 640, 640, True), (1, 6, 2, 130, 130, True), (1, 5, 5, 1, 1, False),
     (3, 4, 4, 129, 1000, True), (1, 16, 16, 16384, 16384, True),
     (1, 2, 2, 640, 128, True), (2, 4, 2, 700, 77, True), (1, 8, 2, 513, 300, True),  # Sq > Sk
+    (2, 8, 2, 1, 700, False), (2, 8, 2, 40, 700, True), (1, 8, 1, 32, 300, True), (3, 4, 2, 128, 128, True),
+    (1, 16, 1, 9, 1000, False), (1, 8, 2, 65, 700, True),  # short GQA queries: packed tiles (the last one is too long)
 ]
 
 
@@ -47,11 +58,15 @@ def test_plan_covers_every_tile_once(kernel, B, Hq, Hkv, Sq, Sk, causal):
     lib.attn_set_option("kernel", kernel)
     plan = lib.attn_plan(B, Hq, Hkv, Sq, Sk, 128, causal, 148)
     g = Hq // Hkv
+    pack = packed_group(Hq, Hkv, Sq) if kernel == 0 else 1
+    tile_rows = TILE // pack
     if kernel == 1:  # one query tile per work item
         assert plan["pair_heads"] == 0 and plan["n_work"] == B * Hq * math.ceil(Sq / TILE)
+    elif pack > 1:   # a tile holds tile_rows query rows of all heads of a KV group
+        assert plan["pair_heads"] == 0 and plan["n_work"] == B * Hkv * math.ceil(math.ceil(Sq / tile_rows) / 2)
     else:
         assert plan["pair_heads"] == (1 if g % 2 == 0 else 0)
-    assert plan["n_q_tiles"] == math.ceil(Sq / TILE) and plan["n_kv_blocks"] == math.ceil(Sk / TILE)
+    assert plan["n_q_tiles"] == math.ceil(Sq / tile_rows) and plan["n_kv_blocks"] == math.ceil(Sk / TILE)
     assert plan["ctas"] == min(148, plan["n_work"])
     seen = {}
     n_work = plan["n_work"]
@@ -62,16 +77,18 @@ def test_plan_covers_every_tile_once(kernel, B, Hq, Hkv, Sq, Sk, causal):
         assert 0 <= it["b"] < B and 0 <= it["hkv"] < Hkv
         for s in (0, 1):
             hq, row0, n = it[f"hq{s}"], it[f"row0_{s}"], it[f"n_blocks_{s}"]
-            assert 0 <= hq < Hq and hq // g == it["hkv"] and row0 % TILE == 0
+            assert 0 <= hq < Hq and hq // g == it["hkv"] and row0 % tile_rows == 0
+            if pack > 1:
+                assert hq == it["hkv"] * g  # the first head of the packed group
             if row0 >= Sq:
                 assert n == 0
                 continue
-            assert n == visible_blocks_brute(row0, Sq, Sk, causal)
+            assert n == visible_blocks_brute(row0, Sq, Sk, causal, tile_rows)
             key = (it["b"], hq, row0)
             assert key not in seen
             seen[key] = w
     if step == 1:
-        assert len(seen) == B * Hq * math.ceil(Sq / TILE)
+        assert len(seen) == B * (Hkv if pack > 1 else Hq) * math.ceil(Sq / tile_rows)
 
 
 def test_causal_items_run_longest_first_inside_a_head():
