@@ -27,6 +27,10 @@ constexpr int kHalfBytes = kTileBytes / 2;        // one [128][64] half tile
 constexpr int kKvSlots = 4;
 constexpr int kThreads = 512;
 constexpr float kRescaleThreshold = 8.0f;  // default log2 units a row maximum may lag behind
+// LSE = m * scale + ln(l) with ln(l) = lg2(l) * ln 2 from the special-function unit (absolute error
+// ~1e-7) and O / l by the approximate reciprocal (2 ulp): the IEEE division and logf subroutines
+// in the epilogue warps cost the softmax warps beside them about 1 % of the whole kernel.
+constexpr float kLn2 = 0.6931471805599453f;
 
 // Registers per thread of each role after the setmaxnreg re-split of the CTA's 64K registers:
 // 8 softmax warps, 4 epilogue warps, 4 other warps; 8 * a + 4 * b + 4 * c must not exceed 2048.
@@ -635,7 +639,7 @@ __device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers
       }
       ++cnt[s];
       tc_fence_after_sync();
-      const float inv_l = l > 0.f ? 1.0f / l : 0.f;  // l = 0: a row without visible keys, O = 0 and LSE = -inf
+      const float inv_l = l > 0.f ? __fdividef(1.0f, l) : 0.f;  // l = 0: a row without visible keys, O = 0 and LSE = -inf
       // the previous TMA store must have finished reading the staging tile
       ok = mbar_wait(&bars.stg_empty[0], (stg_cnt & 1) ^ 1, ctx, kRoleEpilogue | kBarStgEmpty);
       ok = __all_sync(0xffffffffu, ok);
@@ -666,7 +670,7 @@ __device__ __forceinline__ void role_epilogue(const FwdParams& p, const Barriers
       const int row = wk.row0[s] + (row_in_tile >> p.pack_log2);
       const int head = wk.hq[s] + (row_in_tile & ((1 << p.pack_log2) - 1));
       if (p.lse != nullptr && row < p.Sq) {
-        p.lse[(static_cast<size_t>(wk.b) * p.Hq + head) * p.Sq + row] = m_used * p.scale + logf(l);
+        p.lse[(static_cast<size_t>(wk.b) * p.Hq + head) * p.Sq + row] = fmaf(lg2_approx(l), kLn2, m_used * p.scale);
       }
       fence_proxy_async_smem();
       __syncwarp();

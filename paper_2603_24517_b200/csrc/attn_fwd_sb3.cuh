@@ -457,7 +457,7 @@ __device__ __forceinline__ void role_epilogue3(const FwdParams& p, const Bars3& 
     if (l1 > 0.f) l_row += l1 * ex2_approx((m1 - m_fin) * c);
     if (!mbar_wait_warp(&bars.o_full[0], item_cnt & 1, ctx, kRoleEpilogue | kBarOFull)) return;
     tc_fence_after_sync();
-    const float inv_l = l_row > 0.f ? 1.0f / l_row : 0.f;  // a row without visible keys: O = 0, LSE = -inf
+    const float inv_l = l_row > 0.f ? __fdividef(1.0f, l_row) : 0.f;  // a row without visible keys: O = 0, LSE = -inf
     uint8_t* stage = smem + kSmemQ3;
 #pragma unroll
     for (int cc = 0; cc < 4; ++cc) {
@@ -481,7 +481,7 @@ __device__ __forceinline__ void role_epilogue3(const FwdParams& p, const Bars3& 
     if (lane == 0) mbar_arrive(&bars.o_empty[0]);
     const int row = item.row0 + row_in_tile;
     if (p.lse != nullptr && row < p.Sq) {
-      p.lse[(static_cast<size_t>(item.b) * p.Hq + item.hq) * p.Sq + row] = m_fin * p.scale + logf(l_row);
+      p.lse[(static_cast<size_t>(item.b) * p.Hq + item.hq) * p.Sq + row] = fmaf(lg2_approx(l_row), kLn2, m_fin * p.scale);
     }
     fence_proxy_async_smem();
     __syncwarp();
