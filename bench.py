@@ -62,6 +62,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target oracle time of the cpu_baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--set", action="append", default=[], metavar="NAME=VALUE",
+                    help="library option for this run (attn_set_option), e.g. --set kernel=2; repeatable; "
+                         "recorded in config.options")
     return ap.parse_args()
 
 
@@ -287,7 +290,7 @@ def run_ours(args, w):
             "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "Sq": w.Sq, "Sk": w.Sk,
                        "D": w.D, "causal": w.causal, "parallelism": f"replicas x{world}",
                        "l2": f"inputs+outputs {w.algorithmic_bytes / 2**20:.0f} MiB exceed the 126 MB L2; no flush",
-                       "flops_per_step": w.flops},
+                       "flops_per_step": w.flops, "options": args.options},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": args.e2e_steps},
@@ -411,6 +414,7 @@ def run_sweep(args):
     print(json.dumps({
         "metric": METRIC + "_sweep", "unit": UNIT, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
         "protocol": {"warmup_launches": warm, "launches_per_repetition": launches, "repetitions": reps},
+        "options": args.options,
         "geomean": {f: geomean(f) for f in families}, "workloads": entries, "clocks": clocks,
         "gpu_launches": len(entries) * (warm + reps * launches),
     }), flush=True)
@@ -498,8 +502,21 @@ def run_splitkv(args):
 TRAFFIC_BYTES: dict[str, float | None] = {"mha_noncausal_s16384": 522.8e6}
 
 
+def apply_options(args):
+    """Sets the library options given with --set (not for the reference arm, which loads no library)."""
+    args.options = {}
+    for item in args.set:
+        name, _, value = item.partition("=")
+        args.options[name] = int(value)
+    if args.options and args.impl != "reference":
+        import paper_2603_24517_b200 as lib
+        for name, value in args.options.items():
+            lib.attn_set_option(name, value)
+
+
 def main():
     args = parse_args()
+    apply_options(args)
     if args.sweep:
         run_sweep(args)
         return

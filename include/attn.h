@@ -180,6 +180,10 @@ attn_status_t attn_release_host_staging(void);
  *                     of K/V tiles, one score buffer each (default)
  *                 1 = triple score buffer: a CTA runs one query tile with three score tiles
  *                     in flight and two softmax groups that alternate K/V blocks
+ *                 2 = dual query stage on CTA pairs: two CTAs (a cluster) share every
+ *                     tcgen05.mma (M = 256), so a work item is four query tiles and each CTA
+ *                     loads and keeps only half of every K/V tile; same arithmetic per row as
+ *                     "kernel" = 0.  Problems that "gqa_pack" packs run "kernel" = 0.
  */
 attn_status_t attn_set_option(const char* name, int value);
 
@@ -201,9 +205,21 @@ attn_status_t attn_set_option(const char* name, int value);
  * every item has one tile and stage 1 is always unused).
  * Both return ATTN_ERR_SHAPE / ATTN_ERR_UNSUPPORTED like attn_fwd, ATTN_ERR_SHAPE for w
  * out of range.
+ *
+ * With "kernel" = 2 a work item belongs to a pair of CTAs and holds four tiles: `ctas` is
+ * twice the number of pairs, and attn_plan_item_pair gives the item as CTA `rank` (0 = the
+ * leader, 1 = its peer) of the pair sees it, in the layout of attn_plan_item: with
+ * pair_heads = 0 stage s of CTA c holds row tile 4 r + 2 s + c of one head, with
+ * pair_heads = 1 the stages hold two query heads and CTA c row tile 2 r + c.  Both CTAs
+ * report the same n_blocks_s (the two tiles of a stage are multiplied by the same
+ * instructions); a tile whose row0 lies beyond Sq is computed and discarded.
+ * attn_plan_item returns the leader's view.  attn_plan_item_pair returns
+ * ATTN_ERR_UNSUPPORTED when the plan in force is not the pair kernel's.
  */
 attn_status_t attn_plan(int B, int Hq, int Hkv, int Sq, int Sk, int D, int causal, int sm_count, int* plan);
 attn_status_t attn_plan_item(int B, int Hq, int Hkv, int Sq, int Sk, int D, int causal, int w, int* item);
+attn_status_t attn_plan_item_pair(int B, int Hq, int Hkv, int Sq, int Sk, int D, int causal, int w, int rank,
+                                  int* item);
 
 /* Human-readable name of a status code (static storage). */
 const char* attn_status_str(attn_status_t status);

@@ -22,7 +22,7 @@ STATUS_NAMES = {
 }
 EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_strided", "attn_fwd_host", "attn_fwd_noalloc", "attn_merge", "attn_merge_n",
                     "attn_fwd_splitkv", "attn_splitkv_workspace_bytes", "attn_release_host_staging", "attn_set_option",
-                    "attn_plan", "attn_plan_item", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
+                    "attn_plan", "attn_plan_item", "attn_plan_item_pair", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
                     "attn_last_device_status")
 
 _lib = None
@@ -62,6 +62,8 @@ def load_library() -> ctypes.CDLL:
     lib.attn_plan.restype = ci
     lib.attn_plan_item.argtypes = [ci] * 8 + [ctypes.POINTER(ci)]
     lib.attn_plan_item.restype = ci
+    lib.attn_plan_item_pair.argtypes = [ci] * 9 + [ctypes.POINTER(ci)]
+    lib.attn_plan_item_pair.restype = ci
     lib.attn_merge.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
     lib.attn_merge.restype = ci
     lib.attn_merge_n.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, ci, vp]
@@ -220,6 +222,16 @@ def attn_plan_item(B, Hq, Hkv, Sq, Sk, D, causal, w) -> dict:
     st = load_library().attn_plan_item(B, Hq, Hkv, Sq, Sk, D, int(bool(causal)), w, out)
     if st != ATTN_OK:
         raise AttnError(st, "attn_plan_item")
+    keys = ("b", "hkv", "hq0", "hq1", "row0_0", "row0_1", "n_blocks_0", "n_blocks_1")
+    return dict(zip(keys, list(out)))
+
+
+def attn_plan_item_pair(B, Hq, Hkv, Sq, Sk, D, causal, w, rank) -> dict:
+    """Host-only: work item ``w`` of the CTA-pair kernel as CTA ``rank`` of the pair sees it."""
+    out = (ctypes.c_int * 8)()
+    st = load_library().attn_plan_item_pair(B, Hq, Hkv, Sq, Sk, D, int(bool(causal)), w, rank, out)
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_plan_item_pair")
     keys = ("b", "hkv", "hq0", "hq1", "row0_0", "row0_1", "n_blocks_0", "n_blocks_1")
     return dict(zip(keys, list(out)))
 

@@ -9,6 +9,7 @@
 #include "../../include/attn.h"
 #include "attn_fwd_kernel.cuh"
 #include "attn_fwd_sb3.cuh"
+#include "attn_fwd_pair.cuh"
 #include "attn_merge_kernel.cuh"
 
 namespace {
@@ -28,6 +29,7 @@ struct DeviceState {
   bool ready = false;
   bool failed = false;
   int sm_count = 0;
+  int max_pairs = 0;                 // CTA pairs (clusters of two) that can be resident at once
   unsigned int* counters = nullptr;  // [kCounterSlots]
   int* status = nullptr;             // [2]
   std::atomic<unsigned int> next_slot{0};
@@ -46,12 +48,35 @@ DeviceState g_dev[kMaxDevices];
 EncodeTiledFn g_encode = nullptr;
 std::atomic<int> g_opt_scheduler{2};
 std::atomic<int> g_opt_max_ctas{0};
-std::atomic<int> g_opt_kernel{0};  // 0: dual query stage, 1: triple score buffer
+std::atomic<int> g_opt_kernel{0};  // 0: dual query stage, 1: triple score buffer, 2: dual query stage on CTA pairs
 std::atomic<int> g_opt_rescale_threshold{8};
 std::atomic<int> g_opt_split_p{1};
 std::atomic<int> g_opt_overlap_epilogue{1};
 std::atomic<int> g_opt_host_pipeline{1};
 std::atomic<int> g_opt_gqa_pack{1};
+
+// How many clusters of two CTAs of the pair kernel the device holds at once (its shared memory
+// must have been opted in already); never more than one pair per two SMs.
+int resident_pairs(int sm_count) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * (sm_count / 2 > 0 ? sm_count / 2 : 1));
+  cfg.blockDim = dim3(attn::kThreads);
+  cfg.dynamicSmemBytes = attn::pair::kSmemBytes2;
+  cudaLaunchAttribute at;
+  at.id = cudaLaunchAttributeClusterDimension;
+  at.val.clusterDim.x = 2;
+  at.val.clusterDim.y = 1;
+  at.val.clusterDim.z = 1;
+  cfg.attrs = &at;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, attn::pair::attn_fwd_pair_kernel, &cfg) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    n = sm_count / 2;
+  }
+  if (n > sm_count / 2) n = sm_count / 2;
+  return n > 0 ? n : 1;
+}
 
 // Per-device one-time set-up: architecture check, kernel attribute, scheduler counters and
 // status word.  Returns the state or nullptr (with *st set).
@@ -93,12 +118,15 @@ DeviceState* device_state(attn_status_t* st) {
                            attn::kSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(attn::sb3::attn_fwd_sb3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            attn::sb3::kSmemBytes3) != cudaSuccess ||
+      cudaFuncSetAttribute(attn::pair::attn_fwd_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           attn::pair::kSmemBytes2) != cudaSuccess ||
       cudaMalloc(&d.counters, kCounterSlots * sizeof(unsigned int)) != cudaSuccess ||
       cudaMalloc(&d.status, 2 * sizeof(int)) != cudaSuccess ||
       cudaMemset(d.status, 0, 2 * sizeof(int)) != cudaSuccess) {
     *st = ATTN_ERR_CUDA;
     return nullptr;
   }
+  d.max_pairs = resident_pairs(d.sm_count);
   d.ready = true;
   return &d;
 }
@@ -114,13 +142,14 @@ Strides3 contiguous_strides(int S, int H) {
 
 // BF16 tensor seen as 4-D (D, H, S, B) with the given element strides; box = 64 elements x 1 head
 // x 128 rows, 128-byte swizzle, out-of-range rows read as zero and are clipped on store.
-bool make_tensor_map(CUtensorMap* tm, const void* base, int B, int S, int H, Strides3 st, int pack_log2 = 0) {
+bool make_tensor_map(CUtensorMap* tm, const void* base, int B, int S, int H, Strides3 st, int pack_log2 = 0,
+                     unsigned int box_rows = 128) {
   const cuuint64_t dims[4] = {128, static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(S),
                               static_cast<cuuint64_t>(B)};
   const cuuint64_t strides[3] = {static_cast<cuuint64_t>(st.h) * 2, static_cast<cuuint64_t>(st.s) * 2,
                                  static_cast<cuuint64_t>(st.b) * 2};
   // packed query tiles: `group` heads x (128 / group) rows, laid out row-major as (row, head)
-  const cuuint32_t box[4] = {64, 1u << pack_log2, 128u >> pack_log2, 1};
+  const cuuint32_t box[4] = {64, 1u << pack_log2, box_rows >> pack_log2, 1};
   const cuuint32_t elem_strides[4] = {1, 1, 1, 1};
   return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                   elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -160,10 +189,11 @@ void fill_plan(FwdParams* p, int B, int Hq, int Hkv, int Sq, int Sk, int causal)
   // Short query sequences of a GQA group (all of it fits two packed tiles): pack the group's
   // heads into the rows of a tile, so that each KV head is streamed once per row tile pair.
   p->pack_log2 = 0;
-  if (g_opt_gqa_pack.load() != 0 && p->kernel == 0 && p->group >= 2 && p->group <= 16 &&
+  if (g_opt_gqa_pack.load() != 0 && p->kernel != 1 && p->group >= 2 && p->group <= 16 &&
       (p->group & (p->group - 1)) == 0 && Sq <= 2 * (attn::kTile / p->group)) {
     while ((1 << p->pack_log2) < p->group) ++p->pack_log2;
   }
+  if (p->kernel == 2 && p->pack_log2 > 0) p->kernel = 0;  // packed tiles exist in the one-CTA kernel only
   if (p->pack_log2 > 0) {
     p->n_qt = (Sq + (attn::kTile >> p->pack_log2) - 1) / (attn::kTile >> p->pack_log2);
     p->pair_heads = 0;
@@ -173,6 +203,15 @@ void fill_plan(FwdParams* p, int B, int Hq, int Hkv, int Sq, int Sk, int causal)
     p->pair_heads = 0;
     p->items_per_group = p->n_qt;
     p->n_work = B * Hq * p->n_qt;
+  } else if (p->kernel == 2) {  // CTA pairs: four query tiles per work item
+    p->pair_heads = (p->group % 2 == 0) ? 1 : 0;
+    if (p->pair_heads) {
+      p->items_per_group = ((p->n_qt + 1) / 2) * (p->group / 2);
+      p->n_work = B * Hkv * p->items_per_group;
+    } else {
+      p->items_per_group = (p->n_qt + 3) / 4;
+      p->n_work = B * Hq * p->items_per_group;
+    }
   } else {
     p->pair_heads = (p->group % 2 == 0) ? 1 : 0;
     if (p->pair_heads) {
@@ -218,13 +257,26 @@ cudaError_t launch_fwd(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const C
                        const CUtensorMap& tm_o, const FwdParams& p, int grid, cudaStream_t s) {
   if (p.kernel == 1) {
     attn::sb3::attn_fwd_sb3_kernel<<<grid, attn::kThreads, attn::sb3::kSmemBytes3, s>>>(tm_q, tm_k, tm_v, tm_o, p);
+  } else if (p.kernel == 2) {  // grid = 2 x pairs; the cluster shape is a compile-time attribute of the kernel
+    attn::pair::attn_fwd_pair_kernel<<<grid, attn::kThreads, attn::pair::kSmemBytes2, s>>>(tm_q, tm_k, tm_v, tm_o, p);
   } else {
     attn::attn_fwd_kernel<<<grid, attn::kThreads, attn::kSmemBytes, s>>>(tm_q, tm_k, tm_v, tm_o, p);
   }
   return cudaGetLastError();
 }
 
-int plan_grid(const FwdParams& p, int sm_count) {
+int plan_grid(const FwdParams& p, int sm_count, int max_pairs = 0) {
+  if (p.kernel == 2) {  // CTAs come in pairs, one pair per work item in flight
+    int pairs = p.n_work;
+    if (g_opt_scheduler.load() != 0) {
+      int cap = max_pairs > 0 ? max_pairs : sm_count / 2;
+      const int max_ctas = g_opt_max_ctas.load();
+      if (max_ctas > 0 && max_ctas / 2 < cap) cap = max_ctas / 2;
+      if (cap < 1) cap = 1;
+      if (pairs > cap) pairs = cap;
+    }
+    return 2 * pairs;
+  }
   int grid = p.n_work;
   if (g_opt_scheduler.load() != 0) {
     int cap = sm_count;
@@ -272,7 +324,28 @@ attn_status_t attn_plan_item(int B, int Hq, int Hkv, int Sq, int Sk, int D, int 
     return ATTN_OK;
   }
   attn::Work wk;
-  attn::decode_work(p, w, wk);
+  if (p.kernel == 2) {  // the leader CTA's view; attn_plan_item_pair gives either CTA's
+    attn::pair::decode_work_pair(p, w, 0, wk);
+  } else {
+    attn::decode_work(p, w, wk);
+  }
+  item[0] = wk.b; item[1] = wk.hkv; item[2] = wk.hq[0]; item[3] = wk.hq[1];
+  item[4] = wk.row0[0]; item[5] = wk.row0[1]; item[6] = wk.n[0]; item[7] = wk.n[1];
+  return ATTN_OK;
+}
+
+attn_status_t attn_plan_item_pair(int B, int Hq, int Hkv, int Sq, int Sk, int D, int causal, int w, int rank,
+                                  int* item) {
+  if (item == nullptr) return ATTN_ERR_NULL;
+  int dummy = 0;
+  attn_status_t st = check_args(&dummy, &dummy, &dummy, &dummy, nullptr, B, Hq, Hkv, Sq, Sk, D, causal, 1.0f, false);
+  if (st != ATTN_OK) return st;
+  FwdParams p;
+  fill_plan(&p, B, Hq, Hkv, Sq, Sk, causal);
+  if (p.kernel != 2) return ATTN_ERR_UNSUPPORTED;  // the plan in force is not the pair kernel's
+  if (w < 0 || w >= p.n_work || rank < 0 || rank > 1) return ATTN_ERR_SHAPE;
+  attn::Work wk;
+  attn::pair::decode_work_pair(p, w, rank, wk);
   item[0] = wk.b; item[1] = wk.hkv; item[2] = wk.hq[0]; item[3] = wk.hq[1];
   item[4] = wk.row0[0]; item[5] = wk.row0[1]; item[6] = wk.n[0]; item[7] = wk.n[1];
   return ATTN_OK;
@@ -313,7 +386,9 @@ attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, f
   if (causal_off != kDefaultCausalOff) p.off = static_cast<int>(causal_off);
 
   CUtensorMap tm_q, tm_k, tm_v, tm_o;
-  if (!make_tensor_map(&tm_q, q, B, Sq, Hq, sq, p.pack_log2) || !make_tensor_map(&tm_k, k, B, Sk, Hkv, sk) ||
+  // the pair kernel loads K in boxes of 64 keys (each CTA keeps half of a 128-key block)
+  if (!make_tensor_map(&tm_q, q, B, Sq, Hq, sq, p.pack_log2) ||
+      !make_tensor_map(&tm_k, k, B, Sk, Hkv, sk, 0, p.kernel == 2 ? 64 : 128) ||
       !make_tensor_map(&tm_v, v, B, Sk, Hkv, sv) || !make_tensor_map(&tm_o, o, B, Sq, Hq, so, p.pack_log2))
     return ATTN_ERR_CUDA;
 
@@ -321,7 +396,7 @@ attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, f
   p.scale_log2 = scale * 1.4426950408889634f;
   p.lse = lse;
   p.status = dev->status;
-  const int grid = plan_grid(p, dev->sm_count);
+  const int grid = plan_grid(p, dev->sm_count, dev->max_pairs);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (p.dynamic) {
     const unsigned int slot = dev->next_slot.fetch_add(1) % kCounterSlots;
@@ -523,6 +598,8 @@ attn_status_t noalloc_device(NoAllocDevice** out) {
                              attn::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(attn::sb3::attn_fwd_sb3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              attn::sb3::kSmemBytes3) != cudaSuccess ||
+        cudaFuncSetAttribute(attn::pair::attn_fwd_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             attn::pair::kSmemBytes2) != cudaSuccess ||
         cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr)
       return ATTN_ERR_CUDA;
     d.scratch = static_cast<unsigned int*>(ptr);
@@ -549,7 +626,7 @@ attn_status_t attn_fwd_noalloc(const void* q, const void* k, const void* v, void
 
   CUtensorMap tm_q, tm_k, tm_v, tm_o;
   if (!make_tensor_map(&tm_q, q, B, Sq, Hq, contiguous_strides(Sq, Hq), p.pack_log2) ||
-      !make_tensor_map(&tm_k, k, B, Sk, Hkv, contiguous_strides(Sk, Hkv)) ||
+      !make_tensor_map(&tm_k, k, B, Sk, Hkv, contiguous_strides(Sk, Hkv), 0, p.kernel == 2 ? 64 : 128) ||
       !make_tensor_map(&tm_v, v, B, Sk, Hkv, contiguous_strides(Sk, Hkv)) ||
       !make_tensor_map(&tm_o, o, B, Sq, Hq, contiguous_strides(Sq, Hq), p.pack_log2))
     return ATTN_ERR_CUDA;
@@ -596,7 +673,7 @@ attn_status_t attn_set_option(const char* name, int value) {
     return ATTN_OK;
   }
   if (std::strcmp(name, "kernel") == 0) {
-    if (value < 0 || value > 1) return ATTN_ERR_UNSUPPORTED;
+    if (value < 0 || value > 2) return ATTN_ERR_UNSUPPORTED;
     g_opt_kernel.store(value);
     return ATTN_OK;
   }

@@ -115,7 +115,7 @@ SMALL = [
 ]
 
 
-@pytest.fixture(params=[0, 1], ids=["dual_stage", "triple_buffer"])
+@pytest.fixture(params=[0, 1, 2], ids=["dual_stage", "triple_buffer", "cta_pair"])
 def kernel(request):
     """Runs a test once per kernel ("kernel" option of attn_set_option)."""
     lib.attn_set_option("kernel", request.param)

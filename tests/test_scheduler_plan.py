@@ -91,6 +91,50 @@ def test_plan_covers_every_tile_once(kernel, B, Hq, Hkv, Sq, Sk, causal):
         assert len(seen) == B * (Hkv if pack > 1 else Hq) * math.ceil(Sq / tile_rows)
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,causal", CASES)
+def test_pair_plan_covers_every_tile_once(B, Hq, Hkv, Sq, Sk, causal):
+    """CTA-pair kernel: the four tiles of a work item (two stages x two CTAs) cover every query
+    tile exactly once; the two tiles of a stage share a block count, which is what the later of
+    them needs (brute force), so the earlier one never misses a visible block."""
+    lib.attn_set_option("kernel", 2)
+    plan = lib.attn_plan(B, Hq, Hkv, Sq, Sk, 128, causal, 148)
+    g = Hq // Hkv
+    if packed_group(Hq, Hkv, Sq) > 1:  # packed problems keep the one-CTA kernel's plan
+        with pytest.raises(lib.AttnError):
+            lib.attn_plan_item_pair(B, Hq, Hkv, Sq, Sk, 128, causal, 0, 0)
+        return
+    n_qt = math.ceil(Sq / TILE)
+    if g % 2 == 0:
+        assert plan["pair_heads"] == 1 and plan["n_work"] == B * Hkv * math.ceil(n_qt / 2) * (g // 2)
+    else:
+        assert plan["pair_heads"] == 0 and plan["n_work"] == B * Hq * math.ceil(n_qt / 4)
+    assert plan["ctas"] == 2 * min(74, plan["n_work"])
+    seen = set()
+    n_work = plan["n_work"]
+    step = 1 if n_work <= 2048 else 7
+    for w in sorted(set(list(range(0, n_work, step)) + [n_work - 1])):
+        views = [lib.attn_plan_item_pair(B, Hq, Hkv, Sq, Sk, 128, causal, w, r) for r in (0, 1)]
+        assert views[0] == lib.attn_plan_item(B, Hq, Hkv, Sq, Sk, 128, causal, w)
+        for s in (0, 1):
+            a, b = views
+            hq, n = a[f"hq{s}"], a[f"n_blocks_{s}"]
+            assert (b["b"], b["hkv"], b[f"hq{s}"], b[f"n_blocks_{s}"]) == (a["b"], a["hkv"], hq, n)
+            assert 0 <= hq < Hq and hq // g == a["hkv"]
+            assert b[f"row0_{s}"] == a[f"row0_{s}"] + TILE and a[f"row0_{s}"] % (2 * TILE) == 0
+            if a[f"row0_{s}"] >= Sq:
+                assert n == 0
+                continue
+            need = [visible_blocks_brute(v[f"row0_{s}"], Sq, Sk, causal) for v in views if v[f"row0_{s}"] < Sq]
+            assert n == max(need)
+            for v in views:
+                if v[f"row0_{s}"] < Sq:
+                    key = (v["b"], hq, v[f"row0_{s}"])
+                    assert key not in seen
+                    seen.add(key)
+    if step == 1:
+        assert len(seen) == B * Hq * n_qt
+
+
 def test_causal_items_run_longest_first_inside_a_head():
     lib.attn_set_option("kernel", 0)
     B, H, S = 2, 3, 2048
