@@ -11,9 +11,13 @@
 //   O += P V    B = V[128 keys][128 d], N = d:    CTA c holds d 64c .. 64c+63 of all 128 keys (one
 //               MN-major half tile of [128 keys][64 d], 16 KB)
 //
-// Per 128x128x16 step an SM then reads 6 KB (S) or 2 KB (O) of shared memory instead of 8 KB / 4 KB,
-// K/V cross the L2 -> SM path once per 512 query rows instead of once per 256, and the 128 B/clk
-// shared-memory port is no longer the co-limit of the score instructions.
+// Per 128x128x16 step an SM then reads 2 KB of B instead of 4 KB, and K/V cross the L2 -> SM path
+// once per 512 query rows instead of once per 256.  The shared memory and the port bandwidth this
+// frees are spent on P: the softmax warps write P (BF16) into SHARED memory, not over S in tensor
+// memory, so a stage's score tile is free again as soon as its rows have been loaded into
+// registers, and the MMA warp issues S(j+1) = Q K(j+1)^T while the softmax of block j is still
+// running.  A stage's loop is then softmax after softmax, with no wait for P V and Q K^T in
+// between; both matrix products run in the shadow of the exponentials.
 //
 // Roles per CTA as in the one-CTA kernel.  The MMA warp works in the leader CTA (cluster rank 0)
 // only; its commits arrive on the barriers of both CTAs.  What the leader's MMA warp waits for
@@ -29,13 +33,14 @@ namespace attn {
 namespace pair {
 
 constexpr int kKvHalfBytes = kTileBytes / 2;  // this CTA's half of a K or V tile (16 KB)
-constexpr int kKvSlots2 = 8;
+constexpr int kKvSlots2 = 4;
 constexpr int kSmemQ2 = 0;
-constexpr int kSmemKv2 = 2 * kTileBytes;
+constexpr int kSmemP2 = 2 * kTileBytes;             // P_0, P_1: K-major [128 rows][128 keys] as two half tiles
+constexpr int kSmemKv2 = kSmemP2 + 2 * kTileBytes;
 constexpr int kSmemStage2 = kSmemKv2 + kKvSlots2 * kKvHalfBytes;
 constexpr int kSmemStats2 = kSmemStage2 + kTileBytes;
 constexpr int kSmemBars2 = kSmemStats2 + 2 * 2 * kTile * 4;
-constexpr int kNumBars2 = 2 + 2 + 2 * kKvSlots2 + 2 * 10 + 1;
+constexpr int kNumBars2 = 2 + 2 + 2 * kKvSlots2 + 2 * 13 + 1;
 constexpr int kSmemMisc2 = kSmemBars2 + kNumBars2 * 8;
 constexpr int kSmemBytes2 = kSmemMisc2 + 8 + 2 * kMailboxInts * 4;
 static_assert(kSmemBytes2 <= 232448, "shared memory budget of one CTA");
@@ -43,6 +48,9 @@ static_assert(kSmemBytes2 <= 232448, "shared memory budget of one CTA");
 // arrivals per publication on the leader's sched_empty: the leader's MMA lane, and per CTA 8
 // softmax warps and 4 epilogue warps, and the peer's loader
 constexpr int kSchedConsumers2 = 1 + 2 * (8 + 4) + 1;
+
+// wait codes of the barriers this kernel adds (role << 8 | barrier, as in the one-CTA kernel)
+enum : int { kBarSFree = 19, kBarPaEmpty = 20, kBarPbEmpty = 21 };
 
 // Work item `w` of a pair as CTA `rank` sees it.  MHA / odd groups: four consecutive row tiles of
 // one head, stage s of CTA c holds tile 4 r + 2 s + c.  Even GQA groups: the two stages hold two
@@ -126,6 +134,10 @@ __device__ __forceinline__ void mailbox_put_cluster(uint32_t slot_addr, int w, c
 // those that receive arrivals from both CTAs.
 struct PairBars {
   Barriers b;
+  uint64_t* s_free;    // [2]  leader: 4 softmax warps of each CTA have S_s in registers     -> leader's MMA
+  uint64_t* pa_empty;  // [2]  MMA commit: P V over the first 64 keys done (half a of P_s free) -> softmax, both CTAs
+  uint64_t* pb_empty;  // [2]  MMA commit: P V over the last 64 keys done (half b free, O_s quiescent)
+  uint32_t lead_s_free;
   uint32_t lead_q_full;      // [2]  both loaders (expect_tx + TMA bytes)      -> leader's MMA
   uint32_t lead_kv_full;     // [kKvSlots2]
   uint32_t lead_p_half;      // [2]  4 softmax warps of each CTA                -> leader's MMA
@@ -164,13 +176,15 @@ __device__ __forceinline__ void issue_qk2(bool leader, uint32_t tmem_s, uint64_t
   }
 }
 // This CTA's half of a V tile: one MN-major [128 keys][64 d] half tile; 16 keys are 2048 bytes.
-__device__ __forceinline__ void issue_pv2(bool leader, uint32_t tmem_o, uint32_t tmem_p, uint64_t v_desc,
+// P is K-major in shared memory like a Q tile: 16 keys are 32 bytes inside a half tile of 64 keys.
+__device__ __forceinline__ void issue_pv2(bool leader, uint32_t tmem_o, uint64_t p_desc, uint64_t v_desc,
                                           bool accumulate, int kk_begin, int kk_end) {
   if (leader) {
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk) {
       if (kk >= kk_begin && kk < kk_end) {
-        mma_ts_pair(tmem_o, tmem_p + kk * 8, desc_advance(v_desc, kk * 2048), kIdescPV2,
+        const uint32_t p_off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+        mma_ss_pair(tmem_o, desc_advance(p_desc, p_off), desc_advance(v_desc, kk * 2048), kIdescPV2,
                     (accumulate || kk > 0) ? 1u : 0u);
       }
     }
@@ -200,7 +214,7 @@ __device__ __forceinline__ void role_loader2(const FwdParams& p, const PairBars&
     mailbox_put(sched_w, w, wk);  // publication 0 goes to slot 0 of both CTAs, which nobody has used yet
     mailbox_put_cluster(peer_box, w, wk_peer);
     mbar_arrive(&bars.b.sched_full[0]);
-    mbar_arrive_cluster(peer_sched_full);
+    mbar_arrive_cluster_release(peer_sched_full);
   }
   for (int it = 0;; ++it) {
     int w_next = 0;
@@ -221,7 +235,7 @@ __device__ __forceinline__ void role_loader2(const FwdParams& p, const PairBars&
       mailbox_put(sched_w + slot * kMailboxInts, w_next, wk_next);
       mailbox_put_cluster(peer_box + slot * kMailboxInts * 4, w_next, wk_peer);
       mbar_arrive(&bars.b.sched_full[slot]);
-      mbar_arrive_cluster(peer_sched_full + slot * 8);
+      mbar_arrive_cluster_release(peer_sched_full + slot * 8);
     } else {
       // the peer's loader is one more consumer of the mailbox
       const int slot = it & 1;
@@ -275,19 +289,25 @@ __device__ __forceinline__ void role_loader2(const FwdParams& p, const PairBars&
   }
 }
 
-// Leader CTA only.
+// Leader CTA only.  Per K/V block j the order is: S_s(j+1) for both stages (each as soon as the
+// stage's softmax warps have S_s(j) in registers), then P V over the first 64 keys of both stages,
+// then over the last 64 keys.  The softmax warps never wait for a product they have just asked
+// for: S(j+1) is computed while they exponentiate block j.
 __device__ __forceinline__ void role_mma2(const FwdParams& p, const PairBars& bars, uint8_t* smem,
                                           const volatile int* sched_w, WaitCtx ctx, uint32_t tmem, int lane) {
   const bool leader = elect_one();
   const uint32_t smem_base = smem_u32(smem);
   const uint64_t q_desc[2] = {kmajor_desc(smem_base + kSmemQ2), kmajor_desc(smem_base + kSmemQ2 + kTileBytes)};
+  const uint64_t p_desc[2] = {kmajor_desc(smem_base + kSmemP2), kmajor_desc(smem_base + kSmemP2 + kTileBytes)};
   uint32_t kv_cnt = 0;
-  uint32_t q_cnt[2] = {0, 0};
-  uint32_t sp_cnt[2] = {0, 0};
+  uint32_t q_cnt[2] = {0, 0};   // per-stage work items seen (phase of q_full / o_empty)
+  uint32_t qk_cnt[2] = {0, 0};  // per-stage score tiles issued (phase of s_free)
+  uint32_t sp_cnt[2] = {0, 0};  // per-stage K/V blocks whose P has been consumed (phase of p_half / p_full)
   for (int it = 0;; ++it) {
     Work wk;
     const int w = consumer_next_work2(p, bars, sched_w, it, ctx, kRoleMma, lane == 0, wk);
     if (w < 0 || w >= p.n_work) return;
+    // S_s(0) for both stages
     {
       const uint32_t slot = kv_cnt % kKvSlots2, par = (kv_cnt / kKvSlots2) & 1;
       if (!mbar_wait_warp(&bars.b.kv_full[slot], par, ctx, kRoleMma | kBarKvFull)) return;
@@ -296,6 +316,9 @@ __device__ __forceinline__ void role_mma2(const FwdParams& p, const PairBars& ba
       for (int s = 0; s < 2; ++s) {
         if (wk.n[s] > 0) {
           if (!mbar_wait_warp(&bars.b.q_full[s], q_cnt[s] & 1, ctx, kRoleMma | kBarQFull)) return;
+          // the previous score tile of this stage (last block of the previous item) has been read
+          if (!mbar_wait_warp(&bars.s_free[s], (qk_cnt[s] & 1) ^ 1, ctx, kRoleMma | kBarSFree)) return;
+          ++qk_cnt[s];
           tc_fence_after_sync();
           issue_qk2(leader, tmem + s * kTile, q_desc[s], k_desc);
           if (leader) {
@@ -310,17 +333,28 @@ __device__ __forceinline__ void role_mma2(const FwdParams& p, const PairBars& ba
     for (int j = 0; j < wk.nmax; ++j) {
       const uint32_t vslot = kv_cnt % kKvSlots2, vpar = (kv_cnt / kKvSlots2) & 1;
       ++kv_cnt;
-      const bool has_next = (j + 1 < wk.nmax);
-      uint32_t kslot = 0, kpar = 0;
-      if (has_next) {
-        kslot = kv_cnt % kKvSlots2;
-        kpar = (kv_cnt / kKvSlots2) & 1;
+      if (j + 1 < wk.nmax) {  // S_s(j+1), before the softmax warps have finished block j
+        const uint32_t kslot = kv_cnt % kKvSlots2, kpar = (kv_cnt / kKvSlots2) & 1;
         ++kv_cnt;
+        if (!mbar_wait_warp(&bars.b.kv_full[kslot], kpar, ctx, kRoleMma | kBarKvFull)) return;
+        const uint64_t k_desc = kmajor_desc(smem_base + kSmemKv2 + kslot * kKvHalfBytes);
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+          if (j + 1 < wk.n[s]) {
+            if (!mbar_wait_warp(&bars.s_free[s], (qk_cnt[s] & 1) ^ 1, ctx, kRoleMma | kBarSFree)) return;
+            ++qk_cnt[s];
+            tc_fence_after_sync();
+            issue_qk2(leader, tmem + s * kTile, q_desc[s], k_desc);
+            if (leader) {
+              mma_commit_pair(&bars.b.s_full[s]);
+              if (j + 2 == wk.n[s]) mma_commit_pair(&bars.b.q_empty[s]);  // that was the item's last use of Q_s
+            }
+          }
+        }
+        if (leader) mma_commit_pair(&bars.b.kv_empty[kslot]);
       }
       if (!mbar_wait_warp(&bars.b.kv_full[vslot], vpar, ctx, kRoleMma | kBarKvFull)) return;
-      bool k_ready = false;
       const uint64_t v_desc = make_smem_desc_sw128(smem_base + kSmemKv2 + vslot * kKvHalfBytes, kKvHalfBytes, 1024);
-      const uint64_t k_desc = kmajor_desc(smem_base + kSmemKv2 + kslot * kKvHalfBytes);
 #pragma unroll
       for (int s = 0; s < 2; ++s) {
         if (j < wk.n[s]) {
@@ -329,30 +363,24 @@ __device__ __forceinline__ void role_mma2(const FwdParams& p, const PairBars& ba
           }
           if (!mbar_wait_warp(&bars.b.p_half[s], sp_cnt[s] & 1, ctx, kRoleMma | kBarPHalf)) return;
           tc_fence_after_sync();
-          issue_pv2(leader, tmem + 2 * kTile + s * kTile, tmem + s * kTile, v_desc, j > 0, 0, 4);
+          issue_pv2(leader, tmem + 2 * kTile + s * kTile, p_desc[s], v_desc, j > 0, 0, 4);
+          if (leader) mma_commit_pair(&bars.pa_empty[s]);
+        }
+      }
+#pragma unroll
+      for (int s = 0; s < 2; ++s) {
+        if (j < wk.n[s]) {
           if (!mbar_wait_warp(&bars.b.p_full[s], sp_cnt[s] & 1, ctx, kRoleMma | kBarPFull)) return;
           ++sp_cnt[s];
           tc_fence_after_sync();
-          issue_pv2(leader, tmem + 2 * kTile + s * kTile, tmem + s * kTile, v_desc, j > 0, 4, 8);
-          if (leader && j == wk.n[s] - 1) mma_commit_pair(&bars.b.o_full[s]);
-          if (j + 1 < wk.n[s]) {
-            if (!k_ready) {
-              if (!mbar_wait_warp(&bars.b.kv_full[kslot], kpar, ctx, kRoleMma | kBarKvFull)) return;
-              tc_fence_after_sync();
-              k_ready = true;
-            }
-            issue_qk2(leader, tmem + s * kTile, q_desc[s], k_desc);
-            if (leader) {
-              mma_commit_pair(&bars.b.s_full[s]);
-              if (j + 2 == wk.n[s]) mma_commit_pair(&bars.b.q_empty[s]);
-            }
+          issue_pv2(leader, tmem + 2 * kTile + s * kTile, p_desc[s], v_desc, j > 0, 4, 8);
+          if (leader) {
+            mma_commit_pair(&bars.pb_empty[s]);
+            if (j == wk.n[s] - 1) mma_commit_pair(&bars.b.o_full[s]);
           }
         }
       }
-      if (leader) {
-        mma_commit_pair(&bars.b.kv_empty[vslot]);
-        if (has_next) mma_commit_pair(&bars.b.kv_empty[kslot]);
-      }
+      if (leader) mma_commit_pair(&bars.b.kv_empty[vslot]);
     }
 #pragma unroll
     for (int s = 0; s < 2; ++s) {
@@ -362,7 +390,10 @@ __device__ __forceinline__ void role_mma2(const FwdParams& p, const PairBars& ba
 }
 
 // One softmax thread owns one query row of stage `s` of this CTA.  The arithmetic is that of the
-// one-CTA kernel; P is reported to the leader's barriers.
+// one-CTA kernel.  As soon as a block's scores are in registers the score tile is handed back
+// (s_free), so the next block's scores are computed while this one is exponentiated; P goes to
+// shared memory in the layout of a Q tile, each half as soon as the P V that read the previous
+// block's half has completed (pa_empty / pb_empty).
 __device__ __forceinline__ void role_softmax2(const FwdParams& p, const PairBars& bars, uint8_t* smem,
                                               const volatile int* sched_w, WaitCtx ctx, uint32_t tmem, int s,
                                               int row_in_tile, int lane) {
@@ -370,9 +401,13 @@ __device__ __forceinline__ void role_softmax2(const FwdParams& p, const PairBars
   const uint32_t t_s = tmem + lane_sel + s * kTile;
   const uint32_t t_o = tmem + lane_sel + 2 * kTile + s * kTile;
   float* stats = reinterpret_cast<float*>(smem + kSmemStats2) + s * 2 * kTile;
+  // this row of P_s: 128 bytes per half tile, its 16-byte chunks XOR-swizzled with the row index
+  uint8_t* p_row = smem + kSmemP2 + s * kTileBytes + row_in_tile * 128;
+  const uint32_t sw = static_cast<uint32_t>(row_in_tile & 7);
+  const uint32_t s_free = bars.lead_s_free + s * 8;
   const uint32_t p_half = bars.lead_p_half + s * 8, p_full = bars.lead_p_full + s * 8;
   const float c = p.scale_log2;
-  uint32_t s_cnt = 0;
+  uint32_t blk = 0;    // K/V blocks of this stage so far (phases of s_full, pa_empty, pb_empty)
   uint32_t l_cnt = 0;
   for (int it = 0;; ++it) {
     Work wk;
@@ -385,11 +420,10 @@ __device__ __forceinline__ void role_softmax2(const FwdParams& p, const PairBars
     const int tile_clear = p.causal ? min(p.Sk, wk.row0[s] + p.off + 1) : p.Sk;
     float m_used = -INFINITY;
     float l = 0.f;
-    for (int j = 0; j < n; ++j) {
-      bool ok = mbar_wait(&bars.b.s_full[s], s_cnt & 1, ctx, kRoleSoftmax | kBarSFull);
+    for (int j = 0; j < n; ++j, ++blk) {
+      bool ok = mbar_wait(&bars.b.s_full[s], blk & 1, ctx, kRoleSoftmax | kBarSFull);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) return;
-      ++s_cnt;
       tc_fence_after_sync();
       uint32_t xr[kTile];
       tmem_ld_x32(t_s + 0, xr + 0);
@@ -397,6 +431,8 @@ __device__ __forceinline__ void role_softmax2(const FwdParams& p, const PairBars
       tmem_ld_x32(t_s + 64, xr + 64);
       tmem_ld_x32(t_s + 96, xr + 96);
       tmem_wait_ld();
+      tc_fence_before_sync();
+      if (lane == 0) mbar_arrive_cluster(s_free);  // S_s may be overwritten by the next block's scores
 #define X(i) __uint_as_float(xr[(i)])
       if ((j + 1) * kTile > tile_clear) {  // warp-uniform: some element of this block is masked
         const int vis = row_limit - j * kTile;
@@ -422,7 +458,12 @@ __device__ __forceinline__ void role_softmax2(const FwdParams& p, const PairBars
         const float m_new = fmaxf(m_used, m_blk);
         const bool grow = (m_new - m_used) * c > p.rescale_threshold;
         if (__any_sync(0xffffffffu, grow)) {
-          // P V of block j-1 has completed (S of block j was issued after it), so O_s is quiescent
+          // O_s is quiescent once the previous block's P V has completed; this block's is not
+          // issued before this thread's warp has released P
+          ok = mbar_wait(&bars.pb_empty[s], (blk & 1) ^ 1, ctx, kRoleSoftmax | kBarPbEmpty);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) return;
+          tc_fence_after_sync();
           const float alpha = ex2_approx((m_used - m_new) * c);
           m_used = m_new;
           l *= alpha;
@@ -435,6 +476,8 @@ __device__ __forceinline__ void role_softmax2(const FwdParams& p, const PairBars
             for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
             tmem_st_x16(t_o + cc * 16, o);
           }
+          tmem_wait_st();
+          tc_fence_before_sync();
         }
       }
       const float neg_mc = -m_used * c;
@@ -442,41 +485,50 @@ __device__ __forceinline__ void role_softmax2(const FwdParams& p, const PairBars
       const float2 nm2 = make_float2(neg_mc, neg_mc);
       float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t pk[16];
+      for (int h = 0; h < 2; ++h) {
+        // the P V that read this half of the previous block's P must have completed
+        ok = mbar_wait(h == 0 ? &bars.pa_empty[s] : &bars.pb_empty[s], (blk & 1) ^ 1, ctx,
+                       kRoleSoftmax | (h == 0 ? kBarPaEmpty : kBarPbEmpty));
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) return;
 #pragma unroll
-        for (int pr = 0; pr < 16; ++pr) {
-          const int i = cc * 32 + pr * 2;
-          const float2 x = fma2(make_float2(X(i), X(i + 1)), c2, nm2);
-          float2 e;
-          if ((pr & 7) < kExp2PolyPairs) {
-            e = exp2_poly2(x);
-          } else {
-            e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+        for (int ch = 0; ch < 8; ++ch) {  // 16-byte chunk: 8 keys
+          uint32_t pk[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int pr = ch * 4 + q;           // column pair inside the half
+            const int i = h * 64 + pr * 2;
+            const float2 x = fma2(make_float2(X(i), X(i + 1)), c2, nm2);
+            float2 e;
+            if ((pr & 7) < kExp2PolyPairs) {
+              e = exp2_poly2(x);
+            } else {
+              e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+            }
+            if (pr & 1) {
+              lb = add2(lb, e);
+            } else {
+              la = add2(la, e);
+            }
+            pk[q] = pack_bf16x2(e.x, e.y);
           }
-          if (pr & 1) {
-            lb = add2(lb, e);
-          } else {
-            la = add2(la, e);
-          }
-          pk[pr] = pack_bf16x2(e.x, e.y);
+          *reinterpret_cast<uint4*>(p_row + h * kHalfBytes + ((static_cast<uint32_t>(ch) ^ sw) << 4)) =
+              make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
-        tmem_st_x16(t_s + cc * 16, pk);
-        if (cc == 1 && p.split_p) {  // the first 64 keys of P are in tensor memory
-          tmem_wait_st();
-          tc_fence_before_sync();
-          if (lane == 0) mbar_arrive_cluster(p_half);
+        fence_proxy_async_smem();  // the tensor core reads P through the async proxy
+        __syncwarp();
+        if (lane == 0) {
+          if (h == 0) {
+            if (p.split_p) mbar_arrive_cluster(p_half);
+          } else {
+            if (!p.split_p) mbar_arrive_cluster(p_half);
+            mbar_arrive_cluster(p_full);
+          }
         }
       }
 #undef X
       la = add2(la, lb);
       l += la.x + la.y;
-      tmem_wait_st();
-      tc_fence_before_sync();
-      if (lane == 0) {
-        if (!p.split_p) mbar_arrive_cluster(p_half);
-        mbar_arrive_cluster(p_full);
-      }
     }
     bool ok = mbar_wait(&bars.b.l_empty[s], (l_cnt & 1) ^ 1, ctx, kRoleSoftmax | kBarLEmpty);
     ok = __all_sync(0xffffffffu, ok);
@@ -592,6 +644,10 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   bars.b.stg_empty = bars.b.st_full + 2;
   bars.b.sched_full = bars.b.stg_empty + 1;
   bars.b.sched_empty = bars.b.sched_full + 2;
+  bars.s_free = bars.b.sched_empty + 2;
+  bars.pa_empty = bars.s_free + 2;
+  bars.pb_empty = bars.pa_empty + 2;
+  bars.lead_s_free = map_to_cta(smem_u32(bars.s_free), 0);
   bars.lead_q_full = map_to_cta(smem_u32(bars.b.q_full), 0);
   bars.lead_kv_full = map_to_cta(smem_u32(bars.b.kv_full), 0);
   bars.lead_p_half = map_to_cta(smem_u32(bars.b.p_half), 0);
@@ -627,6 +683,9 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       if (i == 0) mbar_init(&bars.b.stg_empty[0], 1);
       mbar_init(&bars.b.sched_full[i], 1);
       mbar_init(&bars.b.sched_empty[i], kSchedConsumers2);
+      mbar_init(&bars.s_free[i], 8);
+      mbar_init(&bars.pa_empty[i], 1);
+      mbar_init(&bars.pb_empty[i], 1);
     }
     for (int i = 0; i < kKvSlots2; ++i) {
       mbar_init(&bars.b.kv_full[i], 2);

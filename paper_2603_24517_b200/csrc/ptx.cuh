@@ -318,13 +318,19 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
 }
-// Arrivals on an mbarrier given by its shared::cluster address (this CTA's or the peer's).
+// Arrivals on an mbarrier given by its shared::cluster address (this CTA's or the peer's).  The
+// plain form orders nothing beyond the CTA: use it where the data travel through tensor memory or
+// TMA (tcgen05 / async-proxy ordering), never for data written with ordinary stores to the peer.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// The same with release semantics at cluster scope (a fence over the thread's earlier writes,
+// those to the peer's shared memory included): pairs with mbar_try_wait_cluster.
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t bar_cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t bar_cluster_addr, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_cluster_addr),
-               "r"(bytes)
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_cluster_addr), "r"(bytes)
                : "memory");
 }
 __device__ __forceinline__ void st_shared_cluster(uint32_t cluster_addr, int value) {
