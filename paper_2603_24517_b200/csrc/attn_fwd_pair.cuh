@@ -19,12 +19,16 @@
 // running.  A stage's loop is then softmax after softmax, with no wait for P V and Q K^T in
 // between; both matrix products run in the shadow of the exponentials.
 //
-// Roles per CTA as in the one-CTA kernel.  The MMA warp works in the leader CTA (cluster rank 0)
-// only; its commits arrive on the barriers of both CTAs.  What the leader's MMA warp waits for
-// (K/V and Q tiles landed, P written, O drained) is counted on the LEADER's barriers: the peer's
-// loader, softmax and epilogue warps arrive there remotely and the peer's TMA loads report their
-// bytes there.  The leader's loader is the pair's tile scheduler and writes each work item into
-// the mailboxes of both CTAs.  No load is multicast: each CTA fetches only what it keeps.
+// Roles per CTA as in the one-CTA kernel, except that there are two MMA warps, one per query stage,
+// and they work in the leader CTA (cluster rank 0) only; their commits arrive on the barriers of
+// both CTAs.  What the leader's MMA warps wait for (K/V and Q tiles landed, S read, P written, O
+// drained) is counted on the LEADER's barriers: the peer's loader, softmax and epilogue warps
+// arrive there remotely and the peer's TMA loads report their bytes there.  Those remote arrivals
+// are plain (the data travel through tensor memory, TMA or proxy-fenced shared memory that the
+// peer's own tensor core reads); only the work-item mailbox, which the leader's loader writes into
+// both CTAs with ordinary stores, is released and acquired at cluster scope: a cluster-scope
+// release on every P hand-over cost a fifth of the kernel's throughput.  No load is multicast: each
+// CTA fetches only what it keeps.
 #pragma once
 
 #include "attn_fwd_kernel.cuh"
@@ -42,15 +46,34 @@ constexpr int kSmemStats2 = kSmemStage2 + kTileBytes;
 constexpr int kSmemBars2 = kSmemStats2 + 2 * 2 * kTile * 4;
 constexpr int kNumBars2 = 2 + 2 + 2 * kKvSlots2 + 2 * 13 + 1;
 constexpr int kSmemMisc2 = kSmemBars2 + kNumBars2 * 8;
-constexpr int kSmemBytes2 = kSmemMisc2 + 8 + 2 * kMailboxInts * 4;
+constexpr int kSmemBytes2 = kSmemMisc2 + 8 + 2 * kMailboxInts * 4 + 8;  // + stage 0's progress word
 static_assert(kSmemBytes2 <= 232448, "shared memory budget of one CTA");
 
-// arrivals per publication on the leader's sched_empty: the leader's MMA lane, and per CTA 8
+// arrivals per publication on the leader's sched_empty: the leader's two MMA warps, and per CTA 8
 // softmax warps and 4 epilogue warps, and the peer's loader
-constexpr int kSchedConsumers2 = 1 + 2 * (8 + 4) + 1;
+constexpr int kSchedConsumers2 = 2 + 2 * (8 + 4) + 1;
 
 // wait codes of the barriers this kernel adds (role << 8 | barrier, as in the one-CTA kernel)
-enum : int { kBarSFree = 19, kBarPaEmpty = 20, kBarPbEmpty = 21 };
+enum : int { kBarSFree = 19, kBarPaEmpty = 20, kBarPbEmpty = 21, kBarProgress = 22 };
+
+// Bounded wait until a shared-memory counter that only grows has reached `target`.
+__device__ __forceinline__ bool wait_counter(const volatile int* counter, int target, WaitCtx ctx, int code) {
+  uint64_t t0 = 0;
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) {
+      if (*counter - target >= 0) return true;
+    }
+    if (*ctx.abort_flag) return false;
+    const uint64_t now = global_timer_ns();
+    if (t0 == 0) t0 = now;
+    if (now - t0 > ctx.limit_ns) {
+      *ctx.abort_flag = 1;
+      if (atomicCAS(ctx.status, 0, code) == 0) ctx.status[1] = static_cast<int>(blockIdx.x);
+      return false;
+    }
+  }
+}
 
 // Work item `w` of a pair as CTA `rank` sees it.  MHA / odd groups: four consecutive row tiles of
 // one head, stage s of CTA c holds tile 4 r + 2 s + c.  Even GQA groups: the two stages hold two
@@ -198,7 +221,7 @@ __device__ __forceinline__ void role_loader2(const FwdParams& p, const PairBars&
                                              volatile int* sched_w, WaitCtx ctx, const CUtensorMap* tm_q,
                                              const CUtensorMap* tm_k, const CUtensorMap* tm_v, int rank) {
   const int n_pairs = static_cast<int>(gridDim.x >> 1);
-  uint32_t kv_cnt = 0;
+  uint32_t kv_base = 0;  // K/V blocks of earlier work items
   uint32_t q_cnt[2] = {0, 0};
   int w = 0;
   Work wk, wk_next, wk_peer;
@@ -251,10 +274,15 @@ __device__ __forceinline__ void role_loader2(const FwdParams& p, const PairBars&
     for (int s = 0; s < 2; ++s) {
       if (wk.n[s] > 0) q_pending |= 1 << s;
     }
-    for (int j = 0; j < wk.nmax; ++j) {
+    // tile order K(0), K(1), V(0), K(2), V(1), ...: the next block's K is asked for before this
+    // block's V, because its scores are computed a block ahead of the P V that reads V
+    for (int t = 0; t <= wk.nmax; ++t) {
       for (int kv = 0; kv < 2; ++kv) {
-        const uint32_t slot = kv_cnt % kKvSlots2;
-        const uint32_t par = (kv_cnt / kKvSlots2) & 1;
+        const int j = kv == 0 ? t : t - 1;  // K(t), then V(t-1)
+        if (j < 0 || j >= wk.nmax) continue;
+        const uint32_t n = kv_base + static_cast<uint32_t>(j);
+        const uint32_t slot = 2 * kv + (n & 1);
+        const uint32_t par = (n >> 1) & 1;
         if (!mbar_wait(&bars.b.kv_empty[slot], par ^ 1, ctx, kRoleLoad | kBarKvEmpty)) return;
         uint8_t* dst = smem + kSmemKv2 + slot * kKvHalfBytes;
         const uint32_t full = bars.lead_kv_full + slot * 8;
@@ -265,8 +293,7 @@ __device__ __forceinline__ void role_loader2(const FwdParams& p, const PairBars&
         } else {        // all 128 keys of the block, head dimension 64 rank .. 64 rank + 63
           tma_load_4d_pair(dst, tm_v, full, rank * 64, wk.hkv, j * kTile, wk.b);
         }
-        ++kv_cnt;
-        if (j == 0 && kv == 0) {
+        if (t == 0 && kv == 0) {
 #pragma unroll
           for (int s = 0; s < 2; ++s) {
             if (q_pending & (1 << s)) {
@@ -282,6 +309,7 @@ __device__ __forceinline__ void role_loader2(const FwdParams& p, const PairBars&
         }
       }
     }
+    kv_base += static_cast<uint32_t>(wk.nmax);
     if (rank == 0) {
       w = w_next;
       wk = wk_next;
@@ -289,103 +317,116 @@ __device__ __forceinline__ void role_loader2(const FwdParams& p, const PairBars&
   }
 }
 
-// Leader CTA only.  Per K/V block j the order is: S_s(j+1) for both stages (each as soon as the
-// stage's softmax warps have S_s(j) in registers), then P V over the first 64 keys of both stages,
-// then over the last 64 keys.  The softmax warps never wait for a product they have just asked
-// for: S(j+1) is computed while they exponentiate block j.
+// Leader CTA only: one MMA warp per query stage (two warps on different sub-partitions), so that the
+// waits and issues of one stage never queue behind the other's in one instruction stream.  Per
+// K/V block j a stage's warp issues, in this order,
+//
+//   S_s(j+1) = Q_s K(j+1)^T   once the stage's softmax warps have S_s(j) in registers
+//   O_s += P_s(j) V(j)        first 64 keys, then last 64 keys, each once it has been written
+//
+// Stage 1 starts an item no less than half a block behind stage 0 (its first score tile waits until
+// the first half of stage 0's first P has been seen; stage 0's warp counts those in a shared-memory
+// word that only grows): one stage's exponentials (special-function unit) then overlap
+// the other's loads, maxima and hand-overs instead of both contending for the same unit at once.
+// K tiles and V tiles live in two rings of two slots each; a slot is free again when BOTH warps
+// have committed it (a warp whose stage does not use a tile waits for it and commits it all the same).
 __device__ __forceinline__ void role_mma2(const FwdParams& p, const PairBars& bars, uint8_t* smem,
-                                          const volatile int* sched_w, WaitCtx ctx, uint32_t tmem, int lane) {
+                                          const volatile int* sched_w, volatile int* progress0, WaitCtx ctx,
+                                          uint32_t tmem, int s, int lane) {
   const bool leader = elect_one();
   const uint32_t smem_base = smem_u32(smem);
-  const uint64_t q_desc[2] = {kmajor_desc(smem_base + kSmemQ2), kmajor_desc(smem_base + kSmemQ2 + kTileBytes)};
-  const uint64_t p_desc[2] = {kmajor_desc(smem_base + kSmemP2), kmajor_desc(smem_base + kSmemP2 + kTileBytes)};
-  uint32_t kv_cnt = 0;
-  uint32_t q_cnt[2] = {0, 0};   // per-stage work items seen (phase of q_full / o_empty)
-  uint32_t qk_cnt[2] = {0, 0};  // per-stage score tiles issued (phase of s_free)
-  uint32_t sp_cnt[2] = {0, 0};  // per-stage K/V blocks whose P has been consumed (phase of p_half / p_full)
+  const uint64_t q_desc = kmajor_desc(smem_base + kSmemQ2 + s * kTileBytes);
+  const uint64_t p_desc = kmajor_desc(smem_base + kSmemP2 + s * kTileBytes);
+  const uint32_t t_s = tmem + s * kTile;
+  const uint32_t t_o = tmem + 2 * kTile + s * kTile;
+  uint32_t kv_base = 0;  // K/V blocks of earlier work items
+  uint32_t q_cnt = 0;    // work items of this stage so far (phase of q_full / o_empty)
+  uint32_t qk_cnt = 0;   // score tiles issued (phase of s_free)
+  uint32_t sp_cnt = 0;   // K/V blocks whose P has been consumed (phase of p_half / p_full)
+  int blk0 = 0;          // stage 0's K/V blocks of earlier work items (stage 1's start signal)
+
+  // waits for tile K(j) (v = 0) or V(j) (v = 1) of the current item; returns its shared memory
+  // address (0: gave up)
+  auto kv_wait = [&](uint32_t v, int j) -> uint32_t {
+    const uint32_t t = kv_base + static_cast<uint32_t>(j), slot = 2 * v + (t & 1), par = (t >> 1) & 1;
+    if (!mbar_wait_warp(&bars.b.kv_full[slot], par, ctx, kRoleMma | kBarKvFull)) return 0u;
+    return smem_base + kSmemKv2 + slot * kKvHalfBytes;
+  };
+  auto kv_release = [&](uint32_t v, int j) {
+    if (leader) mma_commit_pair(&bars.b.kv_empty[2 * v + ((kv_base + static_cast<uint32_t>(j)) & 1)]);
+  };
+  // S_s(j) = Q_s K(j)^T
+  auto scores = [&](int j, int n) -> bool {
+    const uint32_t k_addr = kv_wait(0, j);
+    if (k_addr == 0) return false;
+    // the previous score tile of this stage has been read into registers
+    if (!mbar_wait_warp(&bars.s_free[s], (qk_cnt & 1) ^ 1, ctx, kRoleMma | kBarSFree)) return false;
+    ++qk_cnt;
+    tc_fence_after_sync();
+    issue_qk2(leader, t_s, q_desc, kmajor_desc(k_addr));
+    if (leader) {
+      mma_commit_pair(&bars.b.s_full[s]);
+      if (j == n - 1) mma_commit_pair(&bars.b.q_empty[s]);  // that was the item's last use of Q_s
+    }
+    return true;
+  };
+
   for (int it = 0;; ++it) {
     Work wk;
     const int w = consumer_next_work2(p, bars, sched_w, it, ctx, kRoleMma, lane == 0, wk);
     if (w < 0 || w >= p.n_work) return;
-    // S_s(0) for both stages
-    {
-      const uint32_t slot = kv_cnt % kKvSlots2, par = (kv_cnt / kKvSlots2) & 1;
-      if (!mbar_wait_warp(&bars.b.kv_full[slot], par, ctx, kRoleMma | kBarKvFull)) return;
-      const uint64_t k_desc = kmajor_desc(smem_base + kSmemKv2 + slot * kKvHalfBytes);
-#pragma unroll
-      for (int s = 0; s < 2; ++s) {
-        if (wk.n[s] > 0) {
-          if (!mbar_wait_warp(&bars.b.q_full[s], q_cnt[s] & 1, ctx, kRoleMma | kBarQFull)) return;
-          // the previous score tile of this stage (last block of the previous item) has been read
-          if (!mbar_wait_warp(&bars.s_free[s], (qk_cnt[s] & 1) ^ 1, ctx, kRoleMma | kBarSFree)) return;
-          ++qk_cnt[s];
-          tc_fence_after_sync();
-          issue_qk2(leader, tmem + s * kTile, q_desc[s], k_desc);
-          if (leader) {
-            mma_commit_pair(&bars.b.s_full[s]);
-            if (wk.n[s] == 1) mma_commit_pair(&bars.b.q_empty[s]);
-          }
-        }
+    const int n = wk.n[s];
+    if (n > 0) {
+      if (!mbar_wait_warp(&bars.b.q_full[s], q_cnt & 1, ctx, kRoleMma | kBarQFull)) return;
+      if (s == 1) {  // start behind stage 0: after the first half of its first P of this item
+        bool ok = wait_counter(progress0, blk0 + 1, ctx, kRoleMma | kBarProgress);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) return;
       }
-      if (leader) mma_commit_pair(&bars.b.kv_empty[slot]);
-      ++kv_cnt;
+      if (!scores(0, n)) return;
+    } else if (kv_wait(0, 0) == 0) {
+      return;
     }
+    kv_release(0, 0);
     for (int j = 0; j < wk.nmax; ++j) {
-      const uint32_t vslot = kv_cnt % kKvSlots2, vpar = (kv_cnt / kKvSlots2) & 1;
-      ++kv_cnt;
-      if (j + 1 < wk.nmax) {  // S_s(j+1), before the softmax warps have finished block j
-        const uint32_t kslot = kv_cnt % kKvSlots2, kpar = (kv_cnt / kKvSlots2) & 1;
-        ++kv_cnt;
-        if (!mbar_wait_warp(&bars.b.kv_full[kslot], kpar, ctx, kRoleMma | kBarKvFull)) return;
-        const uint64_t k_desc = kmajor_desc(smem_base + kSmemKv2 + kslot * kKvHalfBytes);
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {
-          if (j + 1 < wk.n[s]) {
-            if (!mbar_wait_warp(&bars.s_free[s], (qk_cnt[s] & 1) ^ 1, ctx, kRoleMma | kBarSFree)) return;
-            ++qk_cnt[s];
-            tc_fence_after_sync();
-            issue_qk2(leader, tmem + s * kTile, q_desc[s], k_desc);
-            if (leader) {
-              mma_commit_pair(&bars.b.s_full[s]);
-              if (j + 2 == wk.n[s]) mma_commit_pair(&bars.b.q_empty[s]);  // that was the item's last use of Q_s
-            }
-          }
+      if (j + 1 < wk.nmax) {
+        // a tile this stage does not use is still handed back only once it has landed: an earlier
+        // commit would be counted for the slot's previous tile, which the other stage may still read
+        if (j + 1 < n) {
+          if (!scores(j + 1, n)) return;
+        } else if (kv_wait(0, j + 1) == 0) {
+          return;
         }
-        if (leader) mma_commit_pair(&bars.b.kv_empty[kslot]);
+        kv_release(0, j + 1);
       }
-      if (!mbar_wait_warp(&bars.b.kv_full[vslot], vpar, ctx, kRoleMma | kBarKvFull)) return;
-      const uint64_t v_desc = make_smem_desc_sw128(smem_base + kSmemKv2 + vslot * kKvHalfBytes, kKvHalfBytes, 1024);
-#pragma unroll
-      for (int s = 0; s < 2; ++s) {
-        if (j < wk.n[s]) {
-          if (j == 0) {  // the previous item's O_s must have left tensor memory in both CTAs
-            if (!mbar_wait_warp(&bars.b.o_empty[s], (q_cnt[s] & 1) ^ 1, ctx, kRoleMma | kBarOEmpty)) return;
-          }
-          if (!mbar_wait_warp(&bars.b.p_half[s], sp_cnt[s] & 1, ctx, kRoleMma | kBarPHalf)) return;
-          tc_fence_after_sync();
-          issue_pv2(leader, tmem + 2 * kTile + s * kTile, p_desc[s], v_desc, j > 0, 0, 4);
-          if (leader) mma_commit_pair(&bars.pa_empty[s]);
+      if (j < n) {
+        const uint32_t v_addr = kv_wait(1, j);
+        if (v_addr == 0) return;
+        const uint64_t v_desc = make_smem_desc_sw128(v_addr, kKvHalfBytes, 1024);
+        if (j == 0) {  // the previous item's O_s must have left tensor memory in both CTAs
+          if (!mbar_wait_warp(&bars.b.o_empty[s], (q_cnt & 1) ^ 1, ctx, kRoleMma | kBarOEmpty)) return;
         }
-      }
-#pragma unroll
-      for (int s = 0; s < 2; ++s) {
-        if (j < wk.n[s]) {
-          if (!mbar_wait_warp(&bars.b.p_full[s], sp_cnt[s] & 1, ctx, kRoleMma | kBarPFull)) return;
-          ++sp_cnt[s];
-          tc_fence_after_sync();
-          issue_pv2(leader, tmem + 2 * kTile + s * kTile, p_desc[s], v_desc, j > 0, 4, 8);
-          if (leader) {
-            mma_commit_pair(&bars.pb_empty[s]);
-            if (j == wk.n[s] - 1) mma_commit_pair(&bars.b.o_full[s]);
-          }
+        if (!mbar_wait_warp(&bars.b.p_half[s], sp_cnt & 1, ctx, kRoleMma | kBarPHalf)) return;
+        tc_fence_after_sync();
+        if (s == 0 && lane == 0) *progress0 = blk0 + j + 1;
+        issue_pv2(leader, t_o, p_desc, v_desc, j > 0, 0, 4);
+        if (leader) mma_commit_pair(&bars.pa_empty[s]);
+        if (!mbar_wait_warp(&bars.b.p_full[s], sp_cnt & 1, ctx, kRoleMma | kBarPFull)) return;
+        ++sp_cnt;
+        tc_fence_after_sync();
+        issue_pv2(leader, t_o, p_desc, v_desc, j > 0, 4, 8);
+        if (leader) {
+          mma_commit_pair(&bars.pb_empty[s]);
+          if (j == n - 1) mma_commit_pair(&bars.b.o_full[s]);
         }
+      } else if (kv_wait(1, j) == 0) {
+        return;
       }
-      if (leader) mma_commit_pair(&bars.b.kv_empty[vslot]);
+      kv_release(1, j);
     }
-#pragma unroll
-    for (int s = 0; s < 2; ++s) {
-      if (wk.n[s] > 0) ++q_cnt[s];
-    }
+    kv_base += static_cast<uint32_t>(wk.nmax);
+    blk0 += wk.n[0];
+    if (n > 0) ++q_cnt;
   }
 }
 
@@ -657,6 +698,7 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kSmemMisc2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kSmemMisc2 + 4);
   volatile int* sched_w = reinterpret_cast<volatile int*>(smem + kSmemMisc2 + 8);
+  volatile int* progress0 = sched_w + 2 * kMailboxInts;
   const WaitCtx ctx{abort_flag, p.status, kWaitLimitNs};
 
   const int tid = threadIdx.x;
@@ -689,9 +731,10 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     }
     for (int i = 0; i < kKvSlots2; ++i) {
       mbar_init(&bars.b.kv_full[i], 2);
-      mbar_init(&bars.b.kv_empty[i], 1);
+      mbar_init(&bars.b.kv_empty[i], 2);  // one commit from each MMA warp
     }
     *abort_flag = bad_align ? 1 : 0;
+    *progress0 = 0;
     fence_mbar_init();
   }
   if (warp == 12) {
@@ -720,8 +763,8 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     tma_store_wait_all0();
   } else {
     reg_dealloc<ATTN_REGS_OTHER>();
-    if (warp == 12) {
-      if (rank == 0 && !bad_align) role_mma2(p, bars, smem, sched_w, ctx, tmem, lane);
+    if (warp == 12 || warp == 14) {  // sub-partitions 0 and 2
+      if (rank == 0 && !bad_align) role_mma2(p, bars, smem, sched_w, progress0, ctx, tmem, (warp - 12) >> 1, lane);
     } else if (warp == 13) {
       if (lane == 0 && !bad_align) {
         role_loader2(p, bars, smem, sched_w, ctx, &tm_q, &tm_k, &tm_v, rank);
