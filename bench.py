@@ -85,18 +85,56 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and clock-event reasons of one GPU through NVML from a thread, about
+    every millisecond, with a host time stamp per sample; stop(t0, t1) keeps the samples taken
+    inside the timed region only.  Falls back to an nvidia-smi child process (25 ms period, all its
+    samples) when the NVML binding is not importable."""
 
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    REASON_BITS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                   "sw_power_cap": 0x4}
 
     def __init__(self, gpu_index: int):
         self.gpu_index = gpu_index
         self.proc = None
         self.file = None
+        self.thread = None
+        self.samples = []  # (host time, sm MHz, power W, reasons mask)
+        self.sm_max = None
+        self._stop = False
+
+    def _nvml_handle(self):
+        import pynvml
+        pynvml.nvmlInit()
+        try:
+            uuid = str(torch.cuda.get_device_properties(self.gpu_index).uuid)
+            return pynvml, pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+        except Exception:
+            return pynvml, pynvml.nvmlDeviceGetHandleByIndex(self.gpu_index)
+
+    def _poll(self, pynvml, handle):
+        while not self._stop:
+            try:
+                mhz = pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM)
+                watts = pynvml.nvmlDeviceGetPowerUsage(handle) / 1000.0
+                mask = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(handle)
+                self.samples.append((time.perf_counter(), float(mhz), watts, int(mask)))
+            except Exception:
+                pass
+            time.sleep(0.001)
 
     def start(self):
+        try:
+            import threading
+            pynvml, handle = self._nvml_handle()
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            self.thread = threading.Thread(target=self._poll, args=(pynvml, handle), daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.thread = None
         try:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
@@ -106,8 +144,21 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.thread is not None:
+            self._stop = True
+            self.thread.join(timeout=2)
+            inside = [x for x in self.samples if (t0 is None or x[0] >= t0) and (t1 is None or x[0] <= t1)]
+            if inside:
+                mask = 0
+                for x in inside:
+                    mask |= x[3]
+                out.update(sm_mhz=statistics.median(x[1] for x in inside), sm_max_mhz=self.sm_max,
+                           reasons=sorted(n for n, bit in self.REASON_BITS.items() if mask & bit),
+                           samples=len(inside), power_w_max=max(x[2] for x in inside),
+                           sm_mhz_min=min(x[1] for x in inside), source="nvml, samples inside the timed region")
+            return out
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -139,7 +190,7 @@ class ClockSampler:
             pass
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons),
-                       samples=len(sm), power_w_max=max(power))
+                       samples=len(sm), power_w_max=max(power), source="nvidia-smi, 25 ms period")
         return out
 
 
@@ -247,13 +298,15 @@ def run_ours(args, w):
         time.sleep(0.15)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin = time.perf_counter()
     e0.record()
     for _ in range(args.steps):
         lib.attn_fwd(q, k, v, o, lse, w.causal, scale)
     e1.record()
     barrier()
+    t_end = time.perf_counter()
     ms_total = e0.elapsed_time(e1)
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     st, code, detail = lib.attn_last_device_status()
     if st != 0:
         raise SystemExit(f"device status {st} code {code:#x} detail {detail}")
