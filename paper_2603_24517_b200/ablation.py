@@ -35,6 +35,7 @@ SWITCHES = [
     ("static round-robin tile scheduler instead of the work counter", {"scheduler": 1}),
     ("one CTA per work item (hardware block scheduler)", {"scheduler": 0}),
     ("triple score buffer kernel instead of dual query stage", {"kernel": 1}),
+    ("CTA-pair kernel (cta_group::2, P through shared memory) instead of dual query stage", {"kernel": 2}),
 ]
 
 
