@@ -304,6 +304,16 @@ def test_triple_buffer_kernel_on_benchmark_workloads(name):
         lib.attn_set_option("kernel", 0)
 
 
+@pytest.mark.parametrize("name", ["mha_noncausal_s16384", "mha_causal_s4096", "gqa4_causal_s8192", "gqa8_noncausal_s4096",
+                                  "long_causal_peaked"])
+def test_cta_pair_kernel_on_benchmark_workloads(name):
+    lib.attn_set_option("kernel", 2)
+    try:
+        test_benchmark_workloads_on_sampled_rows(name)
+    finally:
+        lib.attn_set_option("kernel", 0)
+
+
 def test_decreasing_then_jumping_scores(kernel):
     """Scores that fall for a while and then jump far above everything seen before: the
     reference maxima of consecutive K/V blocks differ by hundreds of log2 units."""
