@@ -184,6 +184,12 @@ attn_status_t attn_release_host_staging(void);
  *                     tcgen05.mma (M = 256), so a work item is four query tiles and each CTA
  *                     loads and keeps only half of every K/V tile; same arithmetic per row as
  *                     "kernel" = 0.  Problems that "gqa_pack" packs run "kernel" = 0.
+ *                 3 = two softmax threads per query row: the default kernel with sixteen softmax
+ *                     warps (each thread exponentiates 64 of a block's 128 keys; partial row
+ *                     maxima are exchanged once per block, partial row sums once per work item)
+ *                     and no separate epilogue warps; the row sum is added up in another order,
+ *                     so results differ from "kernel" = 0 by rounding.  Packed problems run
+ *                     "kernel" = 0.
  */
 attn_status_t attn_set_option(const char* name, int value);
 

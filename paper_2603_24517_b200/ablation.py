@@ -36,6 +36,7 @@ SWITCHES = [
     ("one CTA per work item (hardware block scheduler)", {"scheduler": 0}),
     ("triple score buffer kernel instead of dual query stage", {"kernel": 1}),
     ("CTA-pair kernel (cta_group::2, P through shared memory) instead of dual query stage", {"kernel": 2}),
+    ("two softmax threads per row (sixteen softmax warps, no epilogue warps)", {"kernel": 3}),
 ]
 
 

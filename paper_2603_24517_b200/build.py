@@ -8,7 +8,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libattn_b200.so")
 SOURCES = ["attn_api.cu"]
-HEADERS = ["ptx.cuh", "attn_fwd_kernel.cuh", "attn_fwd_sb3.cuh", "attn_fwd_pair.cuh", "attn_merge_kernel.cuh", os.path.join("..", "..", "include", "attn.h")]
+HEADERS = ["ptx.cuh", "attn_fwd_kernel.cuh", "attn_fwd_sb3.cuh", "attn_fwd_pair.cuh", "attn_fwd_w16.cuh", "attn_merge_kernel.cuh", os.path.join("..", "..", "include", "attn.h")]
 
 
 def _nvcc() -> str:

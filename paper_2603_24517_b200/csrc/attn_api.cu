@@ -10,6 +10,7 @@
 #include "attn_fwd_kernel.cuh"
 #include "attn_fwd_sb3.cuh"
 #include "attn_fwd_pair.cuh"
+#include "attn_fwd_w16.cuh"
 #include "attn_merge_kernel.cuh"
 
 namespace {
@@ -48,7 +49,7 @@ DeviceState g_dev[kMaxDevices];
 EncodeTiledFn g_encode = nullptr;
 std::atomic<int> g_opt_scheduler{2};
 std::atomic<int> g_opt_max_ctas{0};
-std::atomic<int> g_opt_kernel{0};  // 0: dual query stage, 1: triple score buffer, 2: dual query stage on CTA pairs
+std::atomic<int> g_opt_kernel{0};  // 0: dual query stage, 1: triple score buffer, 2: CTA pairs, 3: two softmax threads per row
 std::atomic<int> g_opt_rescale_threshold{8};
 std::atomic<int> g_opt_split_p{1};
 std::atomic<int> g_opt_overlap_epilogue{1};
@@ -120,6 +121,8 @@ DeviceState* device_state(attn_status_t* st) {
                            attn::sb3::kSmemBytes3) != cudaSuccess ||
       cudaFuncSetAttribute(attn::pair::attn_fwd_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            attn::pair::kSmemBytes2) != cudaSuccess ||
+      cudaFuncSetAttribute(attn::w16::attn_fwd_w16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           attn::kSmemBytes) != cudaSuccess ||
       cudaMalloc(&d.counters, kCounterSlots * sizeof(unsigned int)) != cudaSuccess ||
       cudaMalloc(&d.status, 2 * sizeof(int)) != cudaSuccess ||
       cudaMemset(d.status, 0, 2 * sizeof(int)) != cudaSuccess) {
@@ -193,7 +196,7 @@ void fill_plan(FwdParams* p, int B, int Hq, int Hkv, int Sq, int Sk, int causal)
       (p->group & (p->group - 1)) == 0 && Sq <= 2 * (attn::kTile / p->group)) {
     while ((1 << p->pack_log2) < p->group) ++p->pack_log2;
   }
-  if (p->kernel == 2 && p->pack_log2 > 0) p->kernel = 0;  // packed tiles exist in the one-CTA kernel only
+  if (p->kernel >= 2 && p->pack_log2 > 0) p->kernel = 0;  // packed tiles exist in the default kernel only
   if (p->pack_log2 > 0) {
     p->n_qt = (Sq + (attn::kTile >> p->pack_log2) - 1) / (attn::kTile >> p->pack_log2);
     p->pair_heads = 0;
@@ -257,6 +260,8 @@ cudaError_t launch_fwd(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const C
                        const CUtensorMap& tm_o, const FwdParams& p, int grid, cudaStream_t s) {
   if (p.kernel == 1) {
     attn::sb3::attn_fwd_sb3_kernel<<<grid, attn::kThreads, attn::sb3::kSmemBytes3, s>>>(tm_q, tm_k, tm_v, tm_o, p);
+  } else if (p.kernel == 3) {
+    attn::w16::attn_fwd_w16_kernel<<<grid, attn::w16::kThreads16, attn::kSmemBytes, s>>>(tm_q, tm_k, tm_v, tm_o, p);
   } else if (p.kernel == 2) {  // grid = 2 x pairs; the cluster shape is a compile-time attribute of the kernel
     attn::pair::attn_fwd_pair_kernel<<<grid, attn::kThreads, attn::pair::kSmemBytes2, s>>>(tm_q, tm_k, tm_v, tm_o, p);
   } else {
@@ -600,6 +605,8 @@ attn_status_t noalloc_device(NoAllocDevice** out) {
                              attn::sb3::kSmemBytes3) != cudaSuccess ||
         cudaFuncSetAttribute(attn::pair::attn_fwd_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              attn::pair::kSmemBytes2) != cudaSuccess ||
+        cudaFuncSetAttribute(attn::w16::attn_fwd_w16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             attn::kSmemBytes) != cudaSuccess ||
         cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr)
       return ATTN_ERR_CUDA;
     d.scratch = static_cast<unsigned int*>(ptr);
@@ -673,7 +680,7 @@ attn_status_t attn_set_option(const char* name, int value) {
     return ATTN_OK;
   }
   if (std::strcmp(name, "kernel") == 0) {
-    if (value < 0 || value > 2) return ATTN_ERR_UNSUPPORTED;
+    if (value < 0 || value > 3) return ATTN_ERR_UNSUPPORTED;
     g_opt_kernel.store(value);
     return ATTN_OK;
   }

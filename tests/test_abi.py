@@ -68,8 +68,8 @@ def test_options(cdll):
     assert cdll.attn_set_option(None, 1) == 1
     for v in (0, 1, 2):
         assert cdll.attn_set_option(b"scheduler", v) == 0
-    assert cdll.attn_set_option(b"kernel", 3) == 3
-    for v in (2, 1, 0):
+    assert cdll.attn_set_option(b"kernel", 4) == 3
+    for v in (3, 2, 1, 0):
         assert cdll.attn_set_option(b"kernel", v) == 0
     for name, bad, good in ((b"rescale_threshold", 65, 8), (b"split_p", 2, 1), (b"overlap_epilogue", -1, 1)):
         assert cdll.attn_set_option(name, bad) == 3

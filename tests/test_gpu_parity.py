@@ -115,7 +115,7 @@ SMALL = [
 ]
 
 
-@pytest.fixture(params=[0, 1, 2], ids=["dual_stage", "triple_buffer", "cta_pair"])
+@pytest.fixture(params=[0, 1, 2, 3], ids=["dual_stage", "triple_buffer", "cta_pair", "half_row_threads"])
 def kernel(request):
     """Runs a test once per kernel ("kernel" option of attn_set_option)."""
     lib.attn_set_option("kernel", request.param)
@@ -308,6 +308,15 @@ def test_triple_buffer_kernel_on_benchmark_workloads(name):
                                   "long_causal_peaked"])
 def test_cta_pair_kernel_on_benchmark_workloads(name):
     lib.attn_set_option("kernel", 2)
+    try:
+        test_benchmark_workloads_on_sampled_rows(name)
+    finally:
+        lib.attn_set_option("kernel", 0)
+
+
+@pytest.mark.parametrize("name", ["mha_noncausal_s16384", "mha_causal_s4096", "gqa4_causal_s8192", "long_causal_peaked"])
+def test_half_row_kernel_on_benchmark_workloads(name):
+    lib.attn_set_option("kernel", 3)
     try:
         test_benchmark_workloads_on_sampled_rows(name)
     finally:
