@@ -307,6 +307,12 @@ def run_ours(args, w):
     t_end = time.perf_counter()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
+    # NVML's clock reading lags a region of a fraction of a second; the kernel's own cycle counter
+    # over its nanosecond timer gives the clock the last timed launch really ran at
+    in_kernel = lib.attn_last_launch_clock()
+    if clocks is not None and in_kernel is not None:
+        clocks["sm_mhz_last_launch"] = round(in_kernel[0], 1)
+        clocks["last_launch_ms"] = round(in_kernel[1], 4)
     st, code, detail = lib.attn_last_device_status()
     if st != 0:
         raise SystemExit(f"device status {st} code {code:#x} detail {detail}")

@@ -242,6 +242,18 @@ int attn_version(void);
 attn_status_t attn_last_device_status(int* code, int* detail);
 
 /*
+ * attn_last_launch_clock -- the SM clock the most recent launch of the default forward kernel
+ * ("kernel" = 0, through attn_fwd, attn_fwd_strided, attn_fwd_host or attn_fwd_splitkv) actually
+ * ran at on the current device: its first CTA, which lives as long as the launch, reads the SM
+ * cycle counter and the nanosecond timer when it starts and when it ends.  *sm_mhz = cycles /
+ * time, *kernel_ms = that CTA's lifetime.  A measurement aid for benchmarks (the paper reports
+ * throughput on a part whose clock moves under its power limit; Section 4.1): NVML's clock reading
+ * lags a launch of a few milliseconds.  Synchronises the device.  ATTN_ERR_UNSUPPORTED when no such
+ * launch has finished yet.
+ */
+attn_status_t attn_last_launch_clock(double* sm_mhz, double* kernel_ms);
+
+/*
  * attn_merge -- combines two partial attention results that were computed over DISJOINT sets of
  * keys for the same queries (e.g. two attn_fwd calls on the two halves of K and V, non-causal):
  *

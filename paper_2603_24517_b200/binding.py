@@ -22,7 +22,7 @@ STATUS_NAMES = {
 }
 EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_strided", "attn_fwd_host", "attn_fwd_noalloc", "attn_merge", "attn_merge_n",
                     "attn_fwd_splitkv", "attn_splitkv_workspace_bytes", "attn_release_host_staging", "attn_set_option",
-                    "attn_plan", "attn_plan_item", "attn_plan_item_pair", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
+                    "attn_plan", "attn_plan_item", "attn_plan_item_pair", "attn_last_launch_clock", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
                     "attn_last_device_status")
 
 _lib = None
@@ -78,6 +78,8 @@ def load_library() -> ctypes.CDLL:
     lib.attn_status_str.restype = ctypes.c_char_p
     lib.attn_version.argtypes = []
     lib.attn_version.restype = ci
+    lib.attn_last_launch_clock.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    lib.attn_last_launch_clock.restype = ci
     lib.attn_last_device_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.attn_last_device_status.restype = ci
     _lib = lib
@@ -331,6 +333,18 @@ def attn_status_str(status: int) -> str:
 
 def attn_version() -> int:
     return load_library().attn_version()
+
+
+def attn_last_launch_clock():
+    """(SM MHz, milliseconds) of the most recent launch of the default kernel on the current
+    device, or None when there has been none (see include/attn.h)."""
+    mhz, ms = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    st = load_library().attn_last_launch_clock(ctypes.byref(mhz), ctypes.byref(ms))
+    if st == 3:
+        return None
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_last_launch_clock")
+    return mhz.value, ms.value
 
 
 def attn_last_device_status():

@@ -33,6 +33,7 @@ struct DeviceState {
   int max_pairs = 0;                 // CTA pairs (clusters of two) that can be resident at once
   unsigned int* counters = nullptr;  // [kCounterSlots]
   int* status = nullptr;             // [2]
+  unsigned long long* clock_stamps = nullptr;  // [4], see FwdParams
   std::atomic<unsigned int> next_slot{0};
   // attn_fwd_host staging
   void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -125,7 +126,9 @@ DeviceState* device_state(attn_status_t* st) {
                            attn::kSmemBytes) != cudaSuccess ||
       cudaMalloc(&d.counters, kCounterSlots * sizeof(unsigned int)) != cudaSuccess ||
       cudaMalloc(&d.status, 2 * sizeof(int)) != cudaSuccess ||
-      cudaMemset(d.status, 0, 2 * sizeof(int)) != cudaSuccess) {
+      cudaMemset(d.status, 0, 2 * sizeof(int)) != cudaSuccess ||
+      cudaMalloc(&d.clock_stamps, 4 * sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMemset(d.clock_stamps, 0, 4 * sizeof(unsigned long long)) != cudaSuccess) {
     *st = ATTN_ERR_CUDA;
     return nullptr;
   }
@@ -401,6 +404,7 @@ attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, f
   p.scale_log2 = scale * 1.4426950408889634f;
   p.lse = lse;
   p.status = dev->status;
+  p.clock_stamps = dev->clock_stamps;
   const int grid = plan_grid(p, dev->sm_count, dev->max_pairs);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (p.dynamic) {
@@ -855,6 +859,22 @@ const char* attn_status_str(attn_status_t status) {
 }
 
 int attn_version(void) { return 100; }
+
+attn_status_t attn_last_launch_clock(double* sm_mhz, double* kernel_ms) {
+  if (sm_mhz == nullptr || kernel_ms == nullptr) return ATTN_ERR_NULL;
+  attn_status_t st = ATTN_OK;
+  DeviceState* dev = device_state(&st);
+  if (dev == nullptr) return st;
+  unsigned long long h[4] = {0, 0, 0, 0};
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(h, dev->clock_stamps, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return ATTN_ERR_CUDA;
+  if (h[3] <= h[1] || h[2] <= h[0]) return ATTN_ERR_UNSUPPORTED;  // no launch of the default kernel has finished yet
+  const double ns = static_cast<double>(h[3] - h[1]);
+  *kernel_ms = ns * 1e-6;
+  *sm_mhz = static_cast<double>(h[2] - h[0]) / ns * 1e3;
+  return ATTN_OK;
+}
 
 attn_status_t attn_last_device_status(int* code, int* detail) {
   if (code == nullptr || detail == nullptr) return ATTN_ERR_NULL;

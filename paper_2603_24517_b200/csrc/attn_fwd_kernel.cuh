@@ -91,6 +91,8 @@ struct FwdParams {
   float* lse;
   unsigned int* counter;  // dynamic scheduler: next work item - gridDim.x
   int* status;            // [0] code of the first expired wait (0 = none), [1] detail
+  unsigned long long* clock_stamps;  // may be null; the default kernel's CTA 0 writes {clock64, globaltimer} when it
+                                     // starts into [0..1] and when it ends into [2..3]
 };
 
 struct Work {
@@ -729,6 +731,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     return;
   }
   if (tid == 0) {
+    if (blockIdx.x == 0 && p.clock_stamps != nullptr) {  // a persistent CTA lives as long as the launch
+      p.clock_stamps[0] = static_cast<unsigned long long>(clock64());
+      p.clock_stamps[1] = global_timer_ns();
+    }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars.q_full[i], 1);
       mbar_init(&bars.q_empty[i], 1);
@@ -793,6 +799,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   if (warp == 12) {
     tc_fence_after_sync();
     tmem_dealloc(tmem, 512);
+  }
+  if (tid == 0 && blockIdx.x == 0 && p.clock_stamps != nullptr) {
+    p.clock_stamps[2] = static_cast<unsigned long long>(clock64());
+    p.clock_stamps[3] = global_timer_ns();
   }
 }
 

@@ -272,6 +272,13 @@ def test_expired_wait_is_reported_and_the_device_stays_usable():
     check_full(q, k, v, True, SCALE, o, lse)
 
 
+def test_last_launch_clock_is_plausible():
+    q, k, v = make_qkv(2, 4, 4, 2048, 2048, 128, seed=7850)
+    run_gpu(q, k, v, False, SCALE)
+    mhz, ms = lib.attn_last_launch_clock()
+    assert 300.0 < mhz < 2500.0 and 0.0 < ms < 1000.0
+
+
 def test_error_statuses_on_device_tensors():
     q, k, v = (t.cuda() for t in make_qkv(1, 2, 2, 256, 128, 128, seed=7800))
     o = torch.empty_like(q)
