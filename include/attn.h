@@ -242,8 +242,8 @@ int attn_version(void);
 attn_status_t attn_last_device_status(int* code, int* detail);
 
 /*
- * attn_last_launch_clock -- the SM clock the most recent launch of the default forward kernel
- * ("kernel" = 0, through attn_fwd, attn_fwd_strided, attn_fwd_host or attn_fwd_splitkv) actually
+ * attn_last_launch_clock -- the SM clock the most recent launch of a forward kernel ("kernel" =
+ * 0, 2 or 3, through attn_fwd, attn_fwd_strided, attn_fwd_host or attn_fwd_splitkv) actually
  * ran at on the current device: its first CTA, which lives as long as the launch, reads the SM
  * cycle counter and the nanosecond timer when it starts and when it ends.  *sm_mhz = cycles /
  * time, *kernel_ms = that CTA's lifetime.  A measurement aid for benchmarks (the paper reports

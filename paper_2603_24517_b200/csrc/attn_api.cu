@@ -869,7 +869,7 @@ attn_status_t attn_last_launch_clock(double* sm_mhz, double* kernel_ms) {
   if (cudaDeviceSynchronize() != cudaSuccess ||
       cudaMemcpy(h, dev->clock_stamps, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess)
     return ATTN_ERR_CUDA;
-  if (h[3] <= h[1] || h[2] <= h[0]) return ATTN_ERR_UNSUPPORTED;  // no launch of the default kernel has finished yet
+  if (h[3] <= h[1] || h[2] <= h[0]) return ATTN_ERR_UNSUPPORTED;  // no such launch has finished yet
   const double ns = static_cast<double>(h[3] - h[1]);
   *kernel_ms = ns * 1e-6;
   *sm_mhz = static_cast<double>(h[2] - h[0]) / ns * 1e3;

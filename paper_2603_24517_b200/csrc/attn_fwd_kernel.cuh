@@ -91,8 +91,8 @@ struct FwdParams {
   float* lse;
   unsigned int* counter;  // dynamic scheduler: next work item - gridDim.x
   int* status;            // [0] code of the first expired wait (0 = none), [1] detail
-  unsigned long long* clock_stamps;  // may be null; the default kernel's CTA 0 writes {clock64, globaltimer} when it
-                                     // starts into [0..1] and when it ends into [2..3]
+  unsigned long long* clock_stamps;  // may be null; CTA 0 writes {clock64, globaltimer} when it starts into [0..1]
+                                     // and when it ends into [2..3] (not the triple-score-buffer kernel)
 };
 
 struct Work {

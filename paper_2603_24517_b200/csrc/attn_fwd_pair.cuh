@@ -711,6 +711,10 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   const bool bad_align = (smem_u32(smem) & 1023u) != 0;
   if (bad_align && tid == 0 && atomicCAS(p.status, 0, kBadSmemAlign) == 0) p.status[1] = static_cast<int>(blockIdx.x);
   if (tid == 0) {
+    if (blockIdx.x == 0 && p.clock_stamps != nullptr) {
+      p.clock_stamps[0] = static_cast<unsigned long long>(clock64());
+      p.clock_stamps[1] = global_timer_ns();
+    }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars.b.q_full[i], 2);
       mbar_init(&bars.b.q_empty[i], 1);
@@ -783,6 +787,10 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   if (warp == 12) {
     tc_fence_after_sync();
     tmem_dealloc_pair(tmem, 512);
+  }
+  if (tid == 0 && blockIdx.x == 0 && p.clock_stamps != nullptr) {
+    p.clock_stamps[2] = static_cast<unsigned long long>(clock64());
+    p.clock_stamps[3] = global_timer_ns();
   }
 }
 

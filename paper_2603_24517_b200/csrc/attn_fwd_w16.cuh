@@ -247,6 +247,10 @@ attn_fwd_w16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     return;
   }
   if (tid == 0) {
+    if (blockIdx.x == 0 && p.clock_stamps != nullptr) {
+      p.clock_stamps[0] = static_cast<unsigned long long>(clock64());
+      p.clock_stamps[1] = global_timer_ns();
+    }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars.q_full[i], 1);
       mbar_init(&bars.q_empty[i], 1);
@@ -308,6 +312,10 @@ attn_fwd_w16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 16) {
     tc_fence_after_sync();
     tmem_dealloc(tmem, 512);
+  }
+  if (tid == 0 && blockIdx.x == 0 && p.clock_stamps != nullptr) {
+    p.clock_stamps[2] = static_cast<unsigned long long>(clock64());
+    p.clock_stamps[3] = global_timer_ns();
   }
 }
 
