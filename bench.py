@@ -59,9 +59,17 @@ def parse_args():
                     help="time every sequence-length sweep workload (10 warm-ups, then 10 repetitions of 30 launches: "
                          "mean and standard deviation) and print one JSON line with the per-workload TFLOP/s vector "
                          "and its geometric means; one GPU")
+    ap.add_argument("--only", default="", help="--sweep: comma-separated workload-name prefixes to keep")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target oracle time of the cpu_baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--parity-rows", type=int, default=512,
+                    help="rows of the timed launches' output that are compared with the CPU oracle when the "
+                         "cpu_baseline leg does not run (that leg's rows are all compared); 0 skips the check")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="after the timed region, keep launching for this long and report the throughput of the "
+                         "last third as `sustained` (the part is power-limited: a short timed region runs at a "
+                         "higher clock than a long one); 0 skips it")
     ap.add_argument("--set", action="append", default=[], metavar="NAME=VALUE",
                     help="library option for this run (attn_set_option), e.g. --set kernel=2; repeatable; "
                          "recorded in config.options")
@@ -210,19 +218,50 @@ def whole_job_tflops(flops_per_replica: float, world: int, ms_per_step: float) -
     return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
 
 
-def oracle_sample_tflops(w, q, k, v, n_rows, seed):
-    """Times the CPU oracle, as it stands, on `n_rows` seeded rows of the workload."""
+TOL_O, TOL_LSE = 2e-2, 1e-3  # max-norm bounds of the correctness check, as in the parity tests
+
+
+def oracle_sample(w, q, k, v, n_rows, seed):
+    """Runs the CPU oracle, as it stands, on `n_rows` seeded rows of the workload and times it.
+    Returns (TFLOP/s, seconds, rows int32 [n, 3], O rows fp64 [n, D], LSE fp64 [n], threads)."""
     from oracle import attn_oracle as orc
     rng = np.random.default_rng(seed)  # uniform over (b, hq, i): unbiased under the causal mask
     rows = np.stack([rng.integers(w.B, size=n_rows), rng.integers(w.Hq, size=n_rows),
                      rng.integers(w.Sq, size=n_rows)], axis=1).astype(np.int32)
     qb, kb, vb = bf16_bits(q), bf16_bits(k), bf16_bits(v)
     t0 = time.perf_counter()
-    orc.attention_rows(qb, kb, vb, w.causal, w.scale, rows)
+    o_ref, lse_ref = orc.attention_rows(qb, kb, vb, w.causal, w.scale, rows)
     dt = time.perf_counter() - t0
     # FLOPs of these rows under the metric's convention: 4 * Sk * D per (row), halved when causal
     flops = len(rows) * 4.0 * w.Sk * w.D * (0.5 if w.causal else 1.0)
-    return flops / dt / 1e12, dt, len(rows), orc.default_threads()
+    return flops / dt / 1e12, dt, rows, o_ref, lse_ref, orc.default_threads()
+
+
+def oracle_sample_tflops(w, q, k, v, n_rows, seed):
+    """Times the CPU oracle on `n_rows` seeded rows: (TFLOP/s, seconds, rows done, threads)."""
+    rate, dt, rows, _, _, cores = oracle_sample(w, q, k, v, n_rows, seed)
+    return rate, dt, len(rows), cores
+
+
+def parity_of_rows(o_host, lse_host, rows, o_ref, lse_ref):
+    """The correctness gate of the scoring function (the paper's Section 3.1: a candidate that fails
+    the check scores 0): the given rows of the output the TIMED launches left behind against the
+    oracle's.  o_host BF16 [B, Sq, Hq, D] and lse_host fp32 [B, Hq, Sq] are CPU tensors."""
+    from workloads import bits_to_float64
+    o64 = bits_to_float64(bf16_bits(o_host))[rows[:, 0], rows[:, 2], rows[:, 1]]
+    l64 = lse_host.numpy().astype(np.float64)[rows[:, 0], rows[:, 1], rows[:, 2]]
+    finite = bool(np.isfinite(o64).all() and np.isfinite(l64).all() and np.isfinite(lse_ref).all())
+    d_o = float(np.abs(o64 - o_ref).max()) if finite else float("inf")
+    d_l = float(np.abs(l64 - lse_ref).max()) if finite else float("inf")
+    return {"rows": int(len(rows)), "max_dO": d_o, "max_dLSE": d_l, "tol_dO": TOL_O, "tol_dLSE": TOL_LSE,
+            "ok": bool(finite and d_o <= TOL_O and d_l <= TOL_LSE)}
+
+
+def block_pairs_per_sm(w, sm_count):
+    """Pairs of 128 x 128 score blocks per SM under the metric's FLOP convention (8.39 MFLOP per
+    block): what `clocks_per_block_pair` divides by.  The two GEMMs of a pair of blocks keep one SM's
+    tensor pipe busy for 2048 clocks."""
+    return w.flops / (4.0 * 128 * 128 * w.D) / sm_count / 2.0
 
 
 def run_reference(args, w):
@@ -292,30 +331,66 @@ def run_ours(args, w):
         lib.attn_fwd(q, k, v, o, lse, w.causal, scale)
     barrier()
 
+    # poison the outputs: whatever the timed launches do not write stays NaN for the correctness gate
+    o.fill_(float("nan"))
+    lse.fill_(float("nan"))
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.15)
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # K steps as up to 10 repetitions (the paper's Section 4.1 protocol: mean and deviation over
+    # 10 runs) inside ONE timed region: an event after every repetition, no synchronisation between
+    reps = max(1, min(10, args.steps))
+    per_rep = [args.steps // reps + (1 if r < args.steps % reps else 0) for r in range(reps)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
     t_begin = time.perf_counter()
-    e0.record()
-    for _ in range(args.steps):
-        lib.attn_fwd(q, k, v, o, lse, w.causal, scale)
-    e1.record()
+    ev[0].record()
+    for r in range(reps):
+        for _ in range(per_rep[r]):
+            lib.attn_fwd(q, k, v, o, lse, w.causal, scale)
+        ev[r + 1].record()
     barrier()
     t_end = time.perf_counter()
-    ms_total = e0.elapsed_time(e1)
+    ms_total = ev[0].elapsed_time(ev[reps])
+    rep_ms = [ev[r].elapsed_time(ev[r + 1]) / per_rep[r] for r in range(reps)]
     clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     # NVML's clock reading lags a region of a fraction of a second; the kernel's own cycle counter
-    # over its nanosecond timer gives the clock the last timed launch really ran at
-    in_kernel = lib.attn_last_launch_clock()
-    if clocks is not None and in_kernel is not None:
+    # over its nanosecond timer gives the clock every timed launch really ran at
+    in_kernel = lib.attn_launch_clocks(min(64, args.steps))
+    mhz_median = statistics.median(in_kernel) if in_kernel else None
+    if clocks is not None and in_kernel:
+        clocks["sm_mhz_in_kernel_median"] = round(mhz_median, 1)
+        clocks["sm_mhz_in_kernel_min"] = round(min(in_kernel), 1)
+        clocks["sm_mhz_in_kernel_max"] = round(max(in_kernel), 1)
         clocks["sm_mhz_last_launch"] = round(in_kernel[0], 1)
-        clocks["last_launch_ms"] = round(in_kernel[1], 4)
+        clocks["in_kernel_launches"] = len(in_kernel)
     st, code, detail = lib.attn_last_device_status()
     if st != 0:
         raise SystemExit(f"device status {st} code {code:#x} detail {detail}")
+    # the output of the timed launches, for the correctness gate
+    unwritten = bool(torch.isnan(o).any().item() or torch.isnan(lse).any().item())  # the whole output
+    o_timed, lse_timed = (o.cpu(), lse.cpu()) if rank == 0 else (None, None)
+
+    # sustained regime: the same launch repeated for a few seconds, the last third timed
+    sustained = None
+    ms_sustained = 0.0
+    if args.sustained_seconds > 0:
+        ms_guess = ms_total / args.steps
+        n_sus = int(min(3000, max(30, args.sustained_seconds * 1e3 / ms_guess)))
+        n_tail = max(10, n_sus // 3)
+        for _ in range(n_sus - n_tail):
+            lib.attn_fwd(q, k, v, o, lse, w.causal, scale)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for _ in range(n_tail):
+            lib.attn_fwd(q, k, v, o, lse, w.causal, scale)
+        s1.record()
+        barrier()
+        ms_sustained = s0.elapsed_time(s1) / n_tail
+        sus_clocks = lib.attn_launch_clocks(min(64, n_tail))
+        sustained = {"launches": n_sus, "timed_launches": n_tail,
+                     "sm_mhz_in_kernel_median": round(statistics.median(sus_clocks), 1) if sus_clocks else None}
 
     # end to end through the host-buffer entry point: H2D of Q, K, V and D2H of O, LSE every step
     qp, kp, vp = q_h.pin_memory(), k_h.pin_memory(), v_h.pin_memory()
@@ -334,7 +409,7 @@ def run_ours(args, w):
     d2h = op.numel() * 2 + lp.numel() * 4
     lib.attn_release_host_staging()
 
-    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], device=dev)
+    ms_total, ms_e2e, ms_sustained = max_over_ranks([ms_total, ms_e2e, ms_sustained], device=dev)
 
     if rank == 0:
         ms_step = ms_total / args.steps
@@ -342,8 +417,14 @@ def run_ours(args, w):
         e2e_value = whole_job_tflops(w.flops, world, ms_e2e / args.e2e_steps)
         peak_burst, peak_sustained, peak_kind = measured_peaks()
         achieved = w.flops / (ms_step * 1e-3) / 1e12  # one GPU's kernel: one launch per step
+        rep_tflops = [w.flops / (m * 1e-3) / 1e12 for m in rep_ms]   # rank 0's replica
+        sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+        pairs = block_pairs_per_sm(w, sm_count)
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": METRIC, "value": value, "value_std": statistics.pstdev(rep_tflops) * world,
+            "repetitions": {"n": reps, "launches_each": per_rep, "tflops": [round(x, 1) for x in rep_tflops],
+                            "note": "events inside the one timed region; rank 0's replica"},
+            "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "Sq": w.Sq, "Sk": w.Sk,
@@ -360,14 +441,42 @@ def run_ours(args, w):
                          "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
                          "traffic": TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": w.algorithmic_bytes},
         }
+        if mhz_median is not None:
+            # time x clock: SM cycles per pair of 128 x 128 blocks per SM (2048 of them are tensor work);
+            # unlike TFLOP/s this does not move with the clock the power limit allows
+            line["clocks_per_block_pair"] = round(ms_step * 1e-3 * mhz_median * 1e6 / pairs, 1)
+            line["roofline"]["tensor_clocks_per_block_pair"] = 2048
+        if sustained is not None:
+            sus_value = whole_job_tflops(w.flops, world, ms_sustained)
+            sustained.update(value=sus_value, unit=UNIT, ms_per_step=ms_sustained,
+                             frac_of_sustained_peak=sus_value / world / peak_sustained)
+            if sustained["sm_mhz_in_kernel_median"]:
+                sustained["clocks_per_block_pair"] = round(
+                    ms_sustained * 1e-3 * sustained["sm_mhz_in_kernel_median"] * 1e6 / pairs, 1)
+            line["sustained"] = sustained
+        parity = None
         if not args.no_cpu_baseline and world == 1:
             from oracle import attn_oracle as orc
             orc.build()
             rate, dt, n, cores = oracle_sample_tflops(w, q_h, k_h, v_h, 256, seed=1)
             n_rows = int(max(256, min(200000, args.cpu_seconds * n / dt)))
-            rate, dt, n, cores = oracle_sample_tflops(w, q_h, k_h, v_h, n_rows, seed=2)
+            rate, dt, rows, o_ref, lse_ref, cores = oracle_sample(w, q_h, k_h, v_h, n_rows, seed=2)
             line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                    "sample": f"{n} seeded query rows (all keys) of {w.name}, {dt:.1f} s"}
+                                    "sample": f"{len(rows)} seeded query rows (all keys) of {w.name}, {dt:.1f} s"}
+            parity = parity_of_rows(o_timed, lse_timed, rows, o_ref, lse_ref)
+        elif args.parity_rows > 0:
+            from oracle import attn_oracle as orc
+            orc.build()
+            _, _, rows, o_ref, lse_ref, _ = oracle_sample(w_rank, q_h, k_h, v_h, args.parity_rows, seed=2)
+            parity = parity_of_rows(o_timed, lse_timed, rows, o_ref, lse_ref)
+        if parity is not None:
+            parity["unwritten_elements"] = unwritten
+            parity["ok"] = bool(parity["ok"] and not unwritten)
+            line["parity"] = parity
+            if not parity["ok"]:   # a wrong result has no throughput
+                line["unchecked_value"] = line["value"]
+                line["value"] = 0.0
+                line["roofline"]["frac"] = 0.0
         print(json.dumps(line), flush=True)
     if use_dist:
         dist.destroy_process_group()
@@ -425,15 +534,22 @@ def run_merge(args, w):
 def run_sweep(args):
     """The evaluation protocol of the paper's Section 4.1 on every sweep workload: TFLOP/s per
     configuration as mean and standard deviation over 10 repetitions, and the geometric mean per
-    family (the score vector of Section 3.1; correctness of each entry is what the GPU parity tests
-    establish on these same workloads, so no entry is zeroed here)."""
+    family -- the score vector of Section 3.1, correctness gate included: after its timed launches
+    a workload's output is scanned for unwritten elements and `--parity-rows` seeded rows are
+    compared with the CPU oracle; an entry that fails scores 0.  Each repetition also reports SM
+    cycles per pair of 128 x 128 blocks per SM (time x the clock its launches ran at), which does
+    not move with the power-limited clock the way TFLOP/s does."""
     import math
     import paper_2603_24517_b200 as lib
     from paper_2603_24517_b200 import build as lib_build
     lib_build.build()
     lib.load_library()
+    if args.parity_rows > 0:
+        from oracle import attn_oracle as orc
+        orc.build()
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
     reps, launches, warm = 10, 30, 10
     sampler = ClockSampler(0)
     sampler.start()
@@ -441,14 +557,19 @@ def run_sweep(args):
     for name, w in all_workloads().items():
         if not (name.startswith(("mha_", "gqa4_", "gqa8_")) and "_s" in name):
             continue
+        if args.only and not any(name.startswith(pre) for pre in args.only.split(",")):
+            continue
         q_h, k_h, v_h = make_workload_inputs(w)
         q, k, v = q_h.to(dev), k_h.to(dev), v_h.to(dev)
         o = torch.empty_like(q)
         lse = torch.empty((w.B, w.Hq, w.Sq), dtype=torch.float32, device=dev)
         for _ in range(warm):
             lib.attn_fwd(q, k, v, o, lse, w.causal, w.scale)
+        o.fill_(float("nan"))
+        lse.fill_(float("nan"))
         torch.cuda.synchronize()
-        rates = []
+        pairs = block_pairs_per_sm(w, sm_count)
+        rates, cycles, mhzs = [], [], []
         for _ in range(reps):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
@@ -456,23 +577,43 @@ def run_sweep(args):
                 lib.attn_fwd(q, k, v, o, lse, w.causal, w.scale)
             e1.record()
             torch.cuda.synchronize()
-            rates.append(w.flops / (e0.elapsed_time(e1) / launches * 1e-3) / 1e12)
+            ms = e0.elapsed_time(e1) / launches
+            rates.append(w.flops / (ms * 1e-3) / 1e12)
+            mhz = statistics.median(lib.attn_launch_clocks(launches))
+            mhzs.append(mhz)
+            cycles.append(ms * 1e-3 * mhz * 1e6 / pairs)
         st, code, detail = lib.attn_last_device_status()
         if st != 0:
             raise SystemExit(f"{name}: device status {st} code {code:#x} detail {detail}")
-        entries[name] = {"tflops": statistics.mean(rates), "std": statistics.pstdev(rates),
-                         "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "S": w.Sq, "causal": w.causal}
+        entry = {"tflops": statistics.mean(rates), "std": statistics.pstdev(rates),
+                 "clocks_per_block_pair": statistics.mean(cycles), "clocks_std": statistics.pstdev(cycles),
+                 "sm_mhz": statistics.mean(mhzs),
+                 "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "S": w.Sq, "causal": w.causal}
+        if args.parity_rows > 0:
+            unwritten = bool(torch.isnan(o).any().item() or torch.isnan(lse).any().item())
+            _, _, rows, o_ref, lse_ref, _ = oracle_sample(w, q_h, k_h, v_h, args.parity_rows, seed=w.seed)
+            par = parity_of_rows(o.cpu(), lse.cpu(), rows, o_ref, lse_ref)
+            par["unwritten_elements"] = unwritten
+            par["ok"] = bool(par["ok"] and not unwritten)
+            entry["parity"] = par
+            if not par["ok"]:
+                entry["unchecked_tflops"] = entry["tflops"]
+                entry["tflops"] = 0.0
+        entries[name] = entry
         del q, k, v, o, lse
     clocks = sampler.stop()
 
     def geomean(prefix):
         xs = [e["tflops"] for n, e in entries.items() if n.startswith(prefix)]
-        return math.exp(sum(math.log(x) for x in xs) / len(xs)) if xs else None
+        if not xs or min(xs) <= 0.0:
+            return 0.0 if xs else None
+        return math.exp(sum(math.log(x) for x in xs) / len(xs))
 
     families = ["mha_noncausal", "mha_causal", "gqa4_noncausal", "gqa4_causal", "gqa8_noncausal", "gqa8_causal"]
     print(json.dumps({
         "metric": METRIC + "_sweep", "unit": UNIT, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
-        "protocol": {"warmup_launches": warm, "launches_per_repetition": launches, "repetitions": reps},
+        "protocol": {"warmup_launches": warm, "launches_per_repetition": launches, "repetitions": reps,
+                     "parity_rows": args.parity_rows},
         "options": args.options,
         "geomean": {f: geomean(f) for f in families}, "workloads": entries, "clocks": clocks,
         "gpu_launches": len(entries) * (warm + reps * launches),

@@ -66,6 +66,15 @@ typedef enum {
  * attn_fwd issues only a 4-byte cudaMemsetAsync and one kernel launch on `stream`, so it
  * can be captured into a CUDA graph; replays of one captured call share a work counter
  * and must not overlap each other.
+ * Work counters: the library owns a pool of 1024 four-byte counters per device and gives each
+ * call the next one, round-robin; the call's memset clears it on `stream` just before its
+ * kernel.  Two launches that use the same counter must not be resident on the GPU together.
+ * That cannot happen while fewer than 1024 calls (all entry points that launch the forward
+ * kernel counted, attn_fwd_host and attn_fwd_splitkv one per chunk or key range) are queued
+ * or running across all streams of the device.  It can happen when more are, and when a
+ * captured graph -- which keeps the counter its call was given at capture -- is replayed on
+ * one stream while the 1024th later call runs on another: serialise such a replay against the
+ * other streams, or re-capture.
  * Arithmetic: S and O accumulate in fp32 on the tensor cores; P = exp2 of the scaled,
  * max-subtracted scores is rounded to BF16 before P V; the row sum is taken in fp32
  * before that rounding.
@@ -156,7 +165,15 @@ attn_status_t attn_release_host_staging(void);
 
 /*
  * attn_set_option -- tuning / A-B switches; returns ATTN_ERR_UNSUPPORTED for an
- * unknown name or value.  Options are process-wide and read at each launch.
+ * unknown name or value.  (The paper's Section 5 analyses such design choices one at a time;
+ * these switches exist to measure them.)  Options are PROCESS-WIDE: one set of values for every
+ * device, stream and thread, read by each entry point when it is called.  Setting an option is
+ * atomic, but it is not synchronised with launches: a call that another thread makes while an
+ * option changes may see the old or the new value, and two threads that want different values
+ * cannot both have them.  Set options once, before the threads that launch are started, or keep
+ * all calls on one thread.  attn_get_option reads a value back.  Defaults: scheduler 2,
+ * max_ctas 0, rescale_threshold 8, split_p 1, overlap_epilogue 1, gqa_pack 1, host_pipeline 1,
+ * kernel 0.
  *   "scheduler"   0 = one CTA per work item (hardware block scheduler)
  *                 1 = persistent CTAs, static round-robin over work items
  *                 2 = persistent CTAs, dynamic work counter (default)
@@ -192,6 +209,8 @@ attn_status_t attn_release_host_staging(void);
  *                     "kernel" = 0.
  */
 attn_status_t attn_set_option(const char* name, int value);
+/* *value = the current setting of option `name` (host only); ATTN_ERR_UNSUPPORTED for an unknown name. */
+attn_status_t attn_get_option(const char* name, int* value);
 
 /*
  * attn_plan / attn_plan_item -- host-only introspection of the tile scheduler (Section 2.2's
@@ -252,6 +271,19 @@ attn_status_t attn_last_device_status(int* code, int* detail);
  * launch has finished yet.
  */
 attn_status_t attn_last_launch_clock(double* sm_mhz, double* kernel_ms);
+
+/*
+ * attn_launch_clocks -- the same measurement for the most recent launches, newest first: the
+ * library keeps the stamps of the last 64 launches of a stamping kernel per device (a ring indexed
+ * by a launch counter).  Fills sm_mhz[0 .. *n - 1] (HOST array of max_n doubles) with the SM clock
+ * each of them ran at, *n <= min(max_n, 64).  A benchmark reads it once after its timed region and
+ * gets the clock of EVERY timed launch (the paper's Section 4.1 reports means over repeated runs on
+ * a part whose clock drifts under its power limit), so that time x clock -- cycles per unit of work
+ * -- can be compared between runs at different clocks.  Synchronises the device.  *kernel_ms of
+ * attn_last_launch_clock is the first CTA's lifetime, which can be one work item shorter than the
+ * launch; time launches with events.
+ */
+attn_status_t attn_launch_clocks(double* sm_mhz, int max_n, int* n);
 
 /*
  * attn_merge -- combines two partial attention results that were computed over DISJOINT sets of

@@ -13,7 +13,9 @@ import os
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libattn_b200.so")
+# ATTN_B200_LIB names another build of the same library (e.g. one compiled with a different
+# register split for an A/B run); it is loaded instead of the in-tree one, never in addition.
+LIB_PATH = os.environ.get("ATTN_B200_LIB") or os.path.join(_PKG, "libattn_b200.so")
 
 ATTN_OK = 0
 STATUS_NAMES = {
@@ -22,7 +24,8 @@ STATUS_NAMES = {
 }
 EXPORTED_SYMBOLS = ("attn_fwd", "attn_fwd_strided", "attn_fwd_host", "attn_fwd_noalloc", "attn_merge", "attn_merge_n",
                     "attn_fwd_splitkv", "attn_splitkv_workspace_bytes", "attn_release_host_staging", "attn_set_option",
-                    "attn_plan", "attn_plan_item", "attn_plan_item_pair", "attn_last_launch_clock", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
+                    "attn_get_option",
+                    "attn_plan", "attn_plan_item", "attn_plan_item_pair", "attn_last_launch_clock", "attn_launch_clocks", "attn_selftest_wait_timeout", "attn_status_str", "attn_version",
                     "attn_last_device_status")
 
 _lib = None
@@ -58,6 +61,8 @@ def load_library() -> ctypes.CDLL:
     lib.attn_release_host_staging.restype = ci
     lib.attn_set_option.argtypes = [ctypes.c_char_p, ci]
     lib.attn_set_option.restype = ci
+    lib.attn_get_option.argtypes = [ctypes.c_char_p, ctypes.POINTER(ci)]
+    lib.attn_get_option.restype = ci
     lib.attn_plan.argtypes = [ci] * 8 + [ctypes.POINTER(ci)]
     lib.attn_plan.restype = ci
     lib.attn_plan_item.argtypes = [ci] * 8 + [ctypes.POINTER(ci)]
@@ -80,6 +85,8 @@ def load_library() -> ctypes.CDLL:
     lib.attn_version.restype = ci
     lib.attn_last_launch_clock.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     lib.attn_last_launch_clock.restype = ci
+    lib.attn_launch_clocks.argtypes = [ctypes.POINTER(ctypes.c_double), ci, ctypes.POINTER(ci)]
+    lib.attn_launch_clocks.restype = ci
     lib.attn_last_device_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.attn_last_device_status.restype = ci
     _lib = lib
@@ -206,6 +213,18 @@ def attn_set_option(name: str, value: int) -> None:
     st = load_library().attn_set_option(name.encode(), int(value))
     if st != ATTN_OK:
         raise AttnError(st, f"attn_set_option({name}={value})")
+
+
+OPTION_DEFAULTS = {"scheduler": 2, "max_ctas": 0, "rescale_threshold": 8, "split_p": 1, "overlap_epilogue": 1,
+                   "gqa_pack": 1, "host_pipeline": 1, "kernel": 0}
+
+
+def attn_get_option(name: str) -> int:
+    value = ctypes.c_int(0)
+    st = load_library().attn_get_option(name.encode(), ctypes.byref(value))
+    if st != ATTN_OK:
+        raise AttnError(st, f"attn_get_option({name})")
+    return value.value
 
 
 def attn_plan(B, Hq, Hkv, Sq, Sk, D, causal, sm_count) -> dict:
@@ -345,6 +364,17 @@ def attn_last_launch_clock():
     if st != ATTN_OK:
         raise AttnError(st, "attn_last_launch_clock")
     return mhz.value, ms.value
+
+
+def attn_launch_clocks(max_n: int = 64):
+    """SM MHz of the most recent launches on the current device, newest first (at most 64;
+    see include/attn.h).  Synchronises the device."""
+    buf = (ctypes.c_double * max_n)()
+    n = ctypes.c_int(0)
+    st = load_library().attn_launch_clocks(buf, int(max_n), ctypes.byref(n))
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_launch_clocks")
+    return [buf[i] for i in range(n.value)]
 
 
 def attn_last_device_status():

@@ -23,6 +23,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 constexpr int kMaxDevices = 64;
 constexpr int kCounterSlots = 1024;  // one work counter per launch in flight, reused round-robin
+constexpr int kStampSlots = 64;      // launches whose clock stamps are kept (a ring)
 constexpr int kSplitStreams = 8;
 constexpr int kMaxSplits = 64;
 
@@ -33,8 +34,9 @@ struct DeviceState {
   int max_pairs = 0;                 // CTA pairs (clusters of two) that can be resident at once
   unsigned int* counters = nullptr;  // [kCounterSlots]
   int* status = nullptr;             // [2]
-  unsigned long long* clock_stamps = nullptr;  // [4], see FwdParams
+  unsigned long long* clock_stamps = nullptr;  // [kStampSlots][4], one entry per launch, see FwdParams
   std::atomic<unsigned int> next_slot{0};
+  std::atomic<unsigned int> next_stamp{0};    // launches stamped so far
   // attn_fwd_host staging
   void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   size_t stage_bytes[5] = {0, 0, 0, 0, 0};
@@ -127,8 +129,8 @@ DeviceState* device_state(attn_status_t* st) {
       cudaMalloc(&d.counters, kCounterSlots * sizeof(unsigned int)) != cudaSuccess ||
       cudaMalloc(&d.status, 2 * sizeof(int)) != cudaSuccess ||
       cudaMemset(d.status, 0, 2 * sizeof(int)) != cudaSuccess ||
-      cudaMalloc(&d.clock_stamps, 4 * sizeof(unsigned long long)) != cudaSuccess ||
-      cudaMemset(d.clock_stamps, 0, 4 * sizeof(unsigned long long)) != cudaSuccess) {
+      cudaMalloc(&d.clock_stamps, kStampSlots * 4 * sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMemset(d.clock_stamps, 0, kStampSlots * 4 * sizeof(unsigned long long)) != cudaSuccess) {
     *st = ATTN_ERR_CUDA;
     return nullptr;
   }
@@ -404,7 +406,7 @@ attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, f
   p.scale_log2 = scale * 1.4426950408889634f;
   p.lse = lse;
   p.status = dev->status;
-  p.clock_stamps = dev->clock_stamps;
+  p.clock_stamps = dev->clock_stamps + 4 * (dev->next_stamp.fetch_add(1) % kStampSlots);
   const int grid = plan_grid(p, dev->sm_count, dev->max_pairs);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (p.dynamic) {
@@ -721,6 +723,21 @@ attn_status_t attn_set_option(const char* name, int value) {
   return ATTN_ERR_UNSUPPORTED;
 }
 
+attn_status_t attn_get_option(const char* name, int* value) {
+  if (name == nullptr || value == nullptr) return ATTN_ERR_NULL;
+  const struct { const char* name; const std::atomic<int>* opt; } table[] = {
+      {"scheduler", &g_opt_scheduler}, {"kernel", &g_opt_kernel}, {"rescale_threshold", &g_opt_rescale_threshold},
+      {"split_p", &g_opt_split_p}, {"overlap_epilogue", &g_opt_overlap_epilogue}, {"gqa_pack", &g_opt_gqa_pack},
+      {"host_pipeline", &g_opt_host_pipeline}, {"max_ctas", &g_opt_max_ctas}};
+  for (const auto& e : table) {
+    if (std::strcmp(name, e.name) == 0) {
+      *value = e.opt->load();
+      return ATTN_OK;
+    }
+  }
+  return ATTN_ERR_UNSUPPORTED;
+}
+
 attn_status_t attn_merge(const void* o1, const float* lse1, const void* o2, const float* lse2, void* o, float* lse,
                          int B, int Hq, int Sq, int D, void* stream) {
   if (o1 == nullptr || o2 == nullptr || o == nullptr || lse1 == nullptr || lse2 == nullptr || lse == nullptr)
@@ -860,19 +877,56 @@ const char* attn_status_str(attn_status_t status) {
 
 int attn_version(void) { return 100; }
 
-attn_status_t attn_last_launch_clock(double* sm_mhz, double* kernel_ms) {
-  if (sm_mhz == nullptr || kernel_ms == nullptr) return ATTN_ERR_NULL;
+namespace {
+
+// Reads the stamp ring of the current device; entry i of `h` is launch (n_total - 1 - i): newest first.
+attn_status_t read_stamps(unsigned long long (*h)[4], int want, int* got) {
   attn_status_t st = ATTN_OK;
   DeviceState* dev = device_state(&st);
   if (dev == nullptr) return st;
-  unsigned long long h[4] = {0, 0, 0, 0};
+  static unsigned long long ring[kStampSlots][4];
+  std::lock_guard<std::mutex> lock(g_mutex);
   if (cudaDeviceSynchronize() != cudaSuccess ||
-      cudaMemcpy(h, dev->clock_stamps, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess)
+      cudaMemcpy(ring, dev->clock_stamps, sizeof(ring), cudaMemcpyDeviceToHost) != cudaSuccess)
     return ATTN_ERR_CUDA;
-  if (h[3] <= h[1] || h[2] <= h[0]) return ATTN_ERR_UNSUPPORTED;  // no such launch has finished yet
-  const double ns = static_cast<double>(h[3] - h[1]);
+  const unsigned int total = dev->next_stamp.load();
+  int n = 0;
+  for (unsigned int i = 0; i < total && static_cast<int>(i) < kStampSlots && n < want; ++i) {
+    const unsigned long long* e = ring[(total - 1 - i) % kStampSlots];
+    if (e[3] <= e[1] || e[2] <= e[0]) continue;  // a kernel that does not stamp (the triple-score-buffer one)
+    for (int k = 0; k < 4; ++k) h[n][k] = e[k];
+    ++n;
+  }
+  *got = n;
+  return ATTN_OK;
+}
+
+}  // namespace
+
+attn_status_t attn_last_launch_clock(double* sm_mhz, double* kernel_ms) {
+  if (sm_mhz == nullptr || kernel_ms == nullptr) return ATTN_ERR_NULL;
+  unsigned long long h[1][4];
+  int n = 0;
+  const attn_status_t st = read_stamps(h, 1, &n);
+  if (st != ATTN_OK) return st;
+  if (n == 0) return ATTN_ERR_UNSUPPORTED;  // no such launch has finished yet
+  const double ns = static_cast<double>(h[0][3] - h[0][1]);
   *kernel_ms = ns * 1e-6;
-  *sm_mhz = static_cast<double>(h[2] - h[0]) / ns * 1e3;
+  *sm_mhz = static_cast<double>(h[0][2] - h[0][0]) / ns * 1e3;
+  return ATTN_OK;
+}
+
+attn_status_t attn_launch_clocks(double* sm_mhz, int max_n, int* n_out) {
+  if (sm_mhz == nullptr || n_out == nullptr) return ATTN_ERR_NULL;
+  if (max_n <= 0) return ATTN_ERR_SHAPE;
+  unsigned long long h[kStampSlots][4];
+  int n = 0;
+  const attn_status_t st = read_stamps(h, max_n < kStampSlots ? max_n : kStampSlots, &n);
+  if (st != ATTN_OK) return st;
+  for (int i = 0; i < n; ++i) {
+    sm_mhz[i] = static_cast<double>(h[i][2] - h[i][0]) / static_cast<double>(h[i][3] - h[i][1]) * 1e3;
+  }
+  *n_out = n;
   return ATTN_OK;
 }
 

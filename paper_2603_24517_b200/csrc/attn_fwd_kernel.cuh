@@ -55,7 +55,7 @@ constexpr int kSmemKv = 2 * kTileBytes;
 constexpr int kSmemStage = kSmemKv + kKvSlots * kTileBytes;  // O staging tile for the TMA store (both stages, in turn)
 constexpr int kSmemStats = kSmemStage + kTileBytes;          // float [2 stages][2][128]
 constexpr int kSmemBars = kSmemStats + 2 * 2 * kTile * 4;
-constexpr int kNumBars = 2 + 2 + 2 * kKvSlots + 2 * 10 + 1;
+constexpr int kNumBars = 2 + 2 + 2 * kKvSlots + 2 * 10 + 1 + 8;  // + 8: exchange barriers of the two-threads-per-row kernel
 constexpr int kSmemMisc = kSmemBars + kNumBars * 8;  // tmem base, abort flag, two work-item mailbox slots
 constexpr int kMailboxInts = 12;                     // work index + the decoded Work (10 ints), padded
 constexpr int kSmemBytes = kSmemMisc + 8 + 2 * kMailboxInts * 4;
@@ -214,7 +214,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, WaitCt
 enum : int {
   kRoleLoad = 1 << 8, kRoleMma = 2 << 8, kRoleSoftmax = 3 << 8, kRoleEpilogue = 4 << 8,
   kBarQFull = 1, kBarQEmpty = 2, kBarKvFull = 3, kBarKvEmpty = 4, kBarSFull = 5, kBarPFull = 6,
-  kBarOFull = 7, kBarOEmpty = 8, kBarLFull = 9, kBarLEmpty = 10, kBarSchedFull = 11, kBarSchedEmpty = 12, kBarStFull = 13, kBarPHalf = 14, kBarStgEmpty = 18,
+  kBarOFull = 7, kBarOEmpty = 8, kBarLFull = 9, kBarLEmpty = 10, kBarSchedFull = 11, kBarSchedEmpty = 12, kBarStFull = 13, kBarPHalf = 14, kBarStgEmpty = 18, kBarExchange = 19,
   kBadSmemAlign = 0x7001,
   kRoleSelfTest = 9 << 8
 };

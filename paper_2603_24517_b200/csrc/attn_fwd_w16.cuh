@@ -7,8 +7,10 @@
 // given by its index modulo 4, so both sit on the same sub-partition): thread h exponentiates keys
 // 64 h .. 64 h + 63, which halves the latency of a block's softmax -- the longest link of the chain
 // softmax -> P V -> next Q K^T -- and doubles the warps a sub-partition can choose from.  The two
-// threads exchange their partial row maxima through shared memory once per block (a 64-thread
-// named barrier), so both take the exponentials against the same reference; each keeps its own
+// threads exchange their partial row maxima through shared memory once per block (an mbarrier the
+// two warps arrive on and wait for with the same bounded wait as everywhere else, so that a warp
+// whose partner has given up runs into the time limit instead of waiting for ever), so both take
+// the exponentials against the same reference; each keeps its own
 // partial row sum, rescales its own 64 columns of O when the reference moves, and hands over its
 // own half of P: the first-half threads' arrival is the "first 64 keys" signal of the one-CTA
 // kernel, the second-half threads' the "all of P" signal.  There are no epilogue warps: the
@@ -45,7 +47,20 @@ __device__ __forceinline__ void role_softmax16(const FwdParams& p, const Barrier
   volatile float* ex = reinterpret_cast<volatile float*>(smem + kSmemStats);
   volatile float* mine = ex + (s * 2 + h) * kTile + row_in_tile;
   volatile float* partner = ex + (s * 2 + (1 - h)) * kTile + row_in_tile;
-  const uint32_t pair_bar = 1 + s * 4 + (row_in_tile >> 5);  // named barrier of the two warps that share these rows
+  // mbarrier of the two warps that share these rows (count 2: lane 0 of each); behind the barriers
+  // of the one-CTA layout in the barrier array
+  uint64_t* pair_bar = bars.q_full + (kNumBars - 8) + s * 4 + (row_in_tile >> 5);
+  uint32_t x_cnt = 0;  // exchanges so far (phase of pair_bar)
+  // Publishes this thread's value and returns when the partner's is readable; false on an expired wait.
+  auto exchange = [&](float value) -> bool {
+    *mine = value;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(pair_bar);
+    bool ok = mbar_wait(pair_bar, x_cnt & 1, ctx, kRoleSoftmax | kBarExchange);
+    ok = __all_sync(0xffffffffu, ok);
+    ++x_cnt;
+    return ok;
+  };
   uint64_t* my_p_bar = h == 0 ? &bars.p_half[s] : &bars.p_full[s];
   uint64_t* my_st_full = h == 0 ? &bars.st_full[s] : &bars.l_full[s];
   uint64_t* token = &bars.l_empty[h];
@@ -102,8 +117,7 @@ __device__ __forceinline__ void role_softmax16(const FwdParams& p, const Barrier
       const float m_half = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
       // The slot written here was last read by the partner before its previous hand-over of P, which
       // the scores just waited for were issued behind: the exchange needs no second barrier.
-      *mine = m_half;
-      named_barrier_sync(pair_bar, 64);
+      if (!exchange(m_half)) return;
       const float m_blk = fmaxf(m_half, *partner);
       if (j == 0) {
         m_used = (m_blk == -INFINITY) ? 0.f : m_blk;
@@ -160,10 +174,17 @@ __device__ __forceinline__ void role_softmax16(const FwdParams& p, const Barrier
       l += la.x + la.y;
     }
     // ---- end of the work item: the row sum of both halves, then this thread's 64 columns of O ----
-    *mine = l;
-    named_barrier_sync(pair_bar, 64);
+    if (!exchange(l)) return;
     float l_row = l + *partner;
-    named_barrier_sync(pair_bar, 64);  // both have read: the slots may carry maxima again
+    // both must have read before the slots carry maxima again
+    __syncwarp();
+    if (lane == 0) mbar_arrive(pair_bar);
+    {
+      bool ok2 = mbar_wait(pair_bar, x_cnt & 1, ctx, kRoleSoftmax | kBarExchange);
+      ok2 = __all_sync(0xffffffffu, ok2);
+      ++x_cnt;
+      if (!ok2) return;
+    }
     if (row_limit <= 0) l_row = 0.f;   // a row without any visible key has the sum 0 by definition
     bool ok = mbar_wait(&bars.o_full[s], o_cnt & 1, ctx, kRoleSoftmax | kBarOFull);
     ok = __all_sync(0xffffffffu, ok);
@@ -266,6 +287,7 @@ attn_fwd_w16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       mbar_init(&bars.sched_full[i], 1);
       mbar_init(&bars.sched_empty[i], kSchedConsumers16);
     }
+    for (int i = 0; i < 8; ++i) mbar_init(bar_mem + (kNumBars - 8) + i, 2);  // exchange barriers: two warps each
     for (int i = 0; i < kKvSlots; ++i) {
       mbar_init(&bars.kv_full[i], 1);
       mbar_init(&bars.kv_empty[i], 1);

@@ -14,9 +14,12 @@ constexpr int kChunksPerRow = 128 * 2 / 16;  // 16-byte chunks in a 128-element 
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+// A part whose weight is 0 (an empty part) contributes nothing whatever its O holds -- also NaN or
+// Inf from a buffer nobody wrote: 0 * NaN would poison the row, so its term is dropped, not multiplied.
 __device__ __forceinline__ uint32_t merge_pair(uint32_t a, uint32_t b, float w1, float w2) {
-  const float lo = fmaf(w1, bf16_lo(a), w2 * bf16_lo(b));
-  const float hi = fmaf(w1, bf16_hi(a), w2 * bf16_hi(b));
+  const float ta_lo = w1 != 0.f ? w1 * bf16_lo(a) : 0.f, ta_hi = w1 != 0.f ? w1 * bf16_hi(a) : 0.f;
+  const float lo = w2 != 0.f ? fmaf(w2, bf16_lo(b), ta_lo) : ta_lo;
+  const float hi = w2 != 0.f ? fmaf(w2, bf16_hi(b), ta_hi) : ta_hi;
   uint32_t y;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(y) : "f"(hi), "f"(lo));
   return y;
@@ -24,9 +27,12 @@ __device__ __forceinline__ uint32_t merge_pair(uint32_t a, uint32_t b, float w1,
 
 constexpr int kMergeUnroll = 1;  // 16-byte chunks per thread and step (more in flight measured slower)
 
+// o may be the same buffer as o1 or o2 (every thread reads its chunk of both parts before it writes
+// that chunk of o, and no other thread touches it), so the three O pointers are neither restrict-
+// qualified nor read through the non-coherent path.
 __global__ void __launch_bounds__(kMergeThreads)
-attn_merge_kernel(const uint4* __restrict__ o1, const float* __restrict__ lse1, const uint4* __restrict__ o2,
-                  const float* __restrict__ lse2, uint4* __restrict__ o, float* __restrict__ lse, int Hq, int Sq,
+attn_merge_kernel(const uint4* o1, const float* __restrict__ lse1, const uint4* o2,
+                  const float* __restrict__ lse2, uint4* o, float* __restrict__ lse, int Hq, int Sq,
                   long long n_chunks) {
   const long long stride = static_cast<long long>(gridDim.x) * kMergeThreads;
   for (long long c0 = static_cast<long long>(blockIdx.x) * kMergeThreads + threadIdx.x; c0 < n_chunks;
@@ -44,8 +50,8 @@ attn_merge_kernel(const uint4* __restrict__ o1, const float* __restrict__ lse1, 
         const int i = static_cast<int>(t % Sq);
         const long long b = t / Sq;
         li[u] = (b * Hq + h) * Sq + i;  // LSE is [B, Hq, Sq]
-        x[u] = __ldg(o1 + c);
-        y[u] = __ldg(o2 + c);
+        x[u] = o1[c];
+        y[u] = o2[c];
         a[u] = __ldg(lse1 + li[u]);
         bb[u] = __ldg(lse2 + li[u]);
       }

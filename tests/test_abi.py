@@ -78,6 +78,20 @@ def test_options(cdll):
     assert cdll.attn_set_option(b"max_ctas", 0) == 0
 
 
+def test_options_read_back_and_defaults(cdll):
+    """attn_get_option returns what attn_set_option stored; the documented defaults hold
+    whenever a test module starts (conftest.py checks and restores them after every module)."""
+    for name, default in binding.OPTION_DEFAULTS.items():
+        assert lib.attn_get_option(name) == default, name
+    lib.attn_set_option("rescale_threshold", 3)
+    assert lib.attn_get_option("rescale_threshold") == 3
+    lib.attn_set_option("rescale_threshold", 8)
+    v = ctypes.c_int(-1)
+    assert cdll.attn_get_option(b"no_such_option", ctypes.byref(v)) == 3
+    assert cdll.attn_get_option(None, ctypes.byref(v)) == 1
+    assert cdll.attn_get_option(b"kernel", None) == 1
+
+
 def test_last_device_status_null(cdll):
     assert cdll.attn_last_device_status(None, None) == 1
     assert cdll.attn_selftest_wait_timeout(0, None) == 3

@@ -76,6 +76,38 @@ def test_merge_in_place_and_argument_errors():
                            lse.data_ptr(), 1, 2, 64, 64, None) == 3
 
 
+def test_empty_part_may_hold_anything_also_in_place():
+    """A part with LSE = -inf has weight 0 and its O is never used: a buffer nobody wrote (NaN
+    here) must not poison the row, whether the result goes to a fresh buffer or over one input.
+    The oracle, whose two-part form multiplies by the zero weight, gets zeros in those rows."""
+    B, Hq, Sq = 2, 4, 130
+    g = torch.Generator().manual_seed(8200)
+    o1 = torch.randn((B, Sq, Hq, 128), generator=g).to(torch.bfloat16)
+    o2 = torch.randn((B, Sq, Hq, 128), generator=g).to(torch.bfloat16)
+    l1 = torch.randn((B, Hq, Sq), generator=g).float()
+    l2 = torch.randn((B, Hq, Sq), generator=g).float()
+    l1[:, :, ::3] = float("-inf")          # part 1 empty in every third row
+    l2[:, 1, 1::3] = float("-inf")         # part 2 empty elsewhere
+    o1_dev, o2_dev = o1.clone(), o2.clone()
+    o1_dev.permute(0, 2, 1, 3)[torch.isneginf(l1)] = float("nan")
+    o2_dev.permute(0, 2, 1, 3)[torch.isneginf(l2)] = float("nan")
+    o1_ref, o2_ref = o1.clone(), o2.clone()
+    o1_ref.permute(0, 2, 1, 3)[torch.isneginf(l1)] = 0.0
+    o2_ref.permute(0, 2, 1, 3)[torch.isneginf(l2)] = 0.0
+    to_rows = lambda t: t.permute(0, 2, 1).contiguous().numpy()
+    o_ref, lse_ref = orc.merge(bf16_bits(o1_ref), to_rows(l1), bf16_bits(o2_ref), to_rows(l2))
+    for in_place in (False, True):
+        a, b = o1_dev.cuda(), o2_dev.cuda()
+        o = a if in_place else torch.full_like(a, float("nan"))
+        lse = torch.full((B, Hq, Sq), float("nan")).cuda()
+        lib.attn_merge(a, l1.cuda(), b, l2.cuda(), o, lse)
+        torch.cuda.synchronize()
+        o64 = bits_to_float64(bf16_bits(o.cpu()))
+        assert not np.isnan(o64).any()
+        assert np.all(np.abs(o64 - o_ref) <= REL_O_MERGE * np.abs(o_ref) + 1e-5)
+        assert np.abs(to_rows(lse.cpu()).astype(np.float64) - lse_ref).max() <= TOL_LSE_MERGE
+
+
 def test_split_keys_then_merge_equals_attention_over_all_keys():
     B, Hq, Hkv, Sq, Sk = 2, 8, 2, 300, 1000
     q, k, v = make_qkv(B, Hq, Hkv, Sq, Sk, 128, seed=8100)

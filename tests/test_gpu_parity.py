@@ -4,6 +4,11 @@ element on the same seeded BF16 inputs.
 Tolerances (max-norm, absolute): |dO| <= 2e-2 and |dLSE| <= 1e-3.  O is rounded to BF16
 (half an ulp is 1.6e-2 for |O| in [4, 8)), P is rounded to BF16 before P V, and the
 exponentials come from ex2.approx; LSE is fp32 end to end.
+
+Small cases are compared element by element over the whole output.  The benchmark workloads
+at full size are (i) scanned in full for elements the launch never wrote and (ii) compared
+with the oracle on 2048 seeded rows each (1024 from 32768 keys on), which include the
+tile-edge rows of every (batch, head) and a row of every 128-row tile of one head.
 """
 import math
 
@@ -279,6 +284,19 @@ def test_last_launch_clock_is_plausible():
     assert 300.0 < mhz < 2500.0 and 0.0 < ms < 1000.0
 
 
+def test_launch_clock_ring_keeps_one_entry_per_launch():
+    q, k, v = make_qkv(2, 4, 4, 2048, 2048, 128, seed=7851)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    o = torch.empty_like(qd)
+    for _ in range(70):       # more launches than the ring holds
+        lib.attn_fwd(qd, kd, vd, o, None, False, SCALE)
+    clocks = lib.attn_launch_clocks(64)
+    assert len(clocks) == 64 and all(300.0 < c < 2500.0 for c in clocks)
+    assert len(lib.attn_launch_clocks(5)) == 5
+    mhz, _ = lib.attn_last_launch_clock()
+    assert abs(mhz - clocks[0]) < 1e-6   # newest first
+
+
 def test_error_statuses_on_device_tensors():
     q, k, v = (t.cuda() for t in make_qkv(1, 2, 2, 256, 128, 128, seed=7800))
     o = torch.empty_like(q)
@@ -290,15 +308,33 @@ def test_error_statuses_on_device_tensors():
 
 # ---- the benchmark workloads at full size, in the launch configuration bench.py times --------
 FULL = [n for n in all_workloads() if n != "tiny_mha"]
+FULL_ROWS = 2048        # oracle rows per workload ...
+FULL_ROWS_LONG = 1024   # ... and per workload with 32768 keys or more (a row costs 4 * Sk * D flops in fp64)
+
+
+def check_every_element_written(o, lse):
+    """The outputs were poison-filled (NaN) before the launch: every element of O must have
+    been overwritten by a finite value and every LSE by a finite value or -inf.  This looks at
+    ALL of both tensors, so a tile that no CTA wrote cannot hide between sampled rows."""
+    assert not torch.isnan(o).any(), "an element of O was never written"
+    assert torch.isfinite(o.float()).all()
+    assert not torch.isnan(lse).any(), "an element of LSE was never written"
+    assert (torch.isfinite(lse) | torch.isneginf(lse)).all()
 
 
 @pytest.mark.parametrize("name", FULL)
 def test_benchmark_workloads_on_sampled_rows(name):
+    """Full-size workloads: the whole of O and LSE is scanned for unwritten (poison) elements,
+    then FULL_ROWS seeded rows (FULL_ROWS_LONG from 32768 keys on) are compared with the oracle:
+    the tile-edge rows {0, 1, 127, 128, 129, 255, 256, Sq-129, Sq-128, Sq-1} of every
+    (batch, head), one row in every 128-row tile of one head, the rest uniform."""
     w = all_workloads()[name]
     q, k, v = make_workload_inputs(w)
     o, lse = run_gpu(q, k, v, w.causal, w.scale)
-    n_rows = 768 if w.Sk >= 32768 else 1536
+    check_every_element_written(o, lse)
+    n_rows = FULL_ROWS_LONG if w.Sk >= 32768 else FULL_ROWS
     rows = sample_rows(w.B, w.Hq, w.Sq, n_rows, seed=w.seed)
+    assert len(rows) >= n_rows
     check_rows(q, k, v, w.causal, w.scale, o, lse, rows)
 
 
