@@ -698,8 +698,8 @@ def run_splitkv(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of attn_fwd_kernel from the ncu capture
-# summarised in profiles/attn_fwd_kernel_mha_noncausal_s16384_launches.md (404.3 MB + 118.4 MB).
-TRAFFIC_BYTES: dict[str, float | None] = {"mha_noncausal_s16384": 521.4e6}
+# summarised in profiles/attn_fwd_kernel_mha_noncausal_s16384_launches.md (403.3-404.5 MB read + 114.7-118.1 MB written, two launches).
+TRAFFIC_BYTES: dict[str, float | None] = {"mha_noncausal_s16384": 521.3e6}
 
 
 def apply_options(args):
