@@ -406,7 +406,8 @@ attn_status_t fwd_device(const void* q, const void* k, const void* v, void* o, f
   p.scale_log2 = scale * 1.4426950408889634f;
   p.lse = lse;
   p.status = dev->status;
-  p.clock_stamps = dev->clock_stamps + 4 * (dev->next_stamp.fetch_add(1) % kStampSlots);
+  // the triple-score-buffer kernel does not stamp: it takes no ring entry, so every entry counted is one a launch writes
+  p.clock_stamps = p.kernel == 1 ? nullptr : dev->clock_stamps + 4 * (dev->next_stamp.fetch_add(1) % kStampSlots);
   const int grid = plan_grid(p, dev->sm_count, dev->max_pairs);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (p.dynamic) {
@@ -893,7 +894,7 @@ attn_status_t read_stamps(unsigned long long (*h)[4], int want, int* got) {
   int n = 0;
   for (unsigned int i = 0; i < total && static_cast<int>(i) < kStampSlots && n < want; ++i) {
     const unsigned long long* e = ring[(total - 1 - i) % kStampSlots];
-    if (e[3] <= e[1] || e[2] <= e[0]) continue;  // a kernel that does not stamp (the triple-score-buffer one)
+    if (e[3] <= e[1] || e[2] <= e[0]) continue;  // still running, or a launch that ended on an expired wait
     for (int k = 0; k < 4; ++k) h[n][k] = e[k];
     ++n;
   }
