@@ -98,6 +98,30 @@ def test_last_device_status_null(cdll):
     assert cdll.attn_selftest_wait_timeout(5000, None) == 3
 
 
+def test_clock_ring_argument_errors_need_no_device(cdll):
+    n = ctypes.c_int(0)
+    buf = (ctypes.c_double * 4)()
+    assert cdll.attn_launch_clocks(None, 4, ctypes.byref(n)) == 1     # ATTN_ERR_NULL
+    assert cdll.attn_launch_clocks(buf, 4, None) == 1
+    assert cdll.attn_launch_clocks(buf, 0, ctypes.byref(n)) == 2      # ATTN_ERR_SHAPE
+    assert cdll.attn_last_launch_clock(None, None) == 1
+
+
+def test_variant_build_reports_spills_and_exports_the_abi(tmp_path):
+    """Another register split is a build of its own beside the in-tree library (how the register-split
+    rows of the ablation are made): it must export the whole ABI and report ptxas's spill figures."""
+    out = str(tmp_path / "libattn_b200_176_80_80.so")
+    info = lib_build.build_variant(out, ["-DATTN_REGS_SOFTMAX=176", "-DATTN_REGS_EPILOGUE=80", "-DATTN_REGS_OTHER=80"])
+    assert info["path"] == out and os.path.exists(out)
+    assert isinstance(info["spill_store_bytes"], int) and isinstance(info["spill_load_bytes"], int)
+    other = ctypes.CDLL(out)
+    for name in binding.EXPORTED_SYMBOLS:
+        assert hasattr(other, name)
+    with pytest.raises(RuntimeError):   # 8 a + 4 b + 4 c > 2048 is refused at compile time (static_assert)
+        lib_build.build_variant(str(tmp_path / "bad.so"), ["-DATTN_REGS_SOFTMAX=200", "-DATTN_REGS_EPILOGUE=128",
+                                                           "-DATTN_REGS_OTHER=128"])
+
+
 def test_missing_library_is_loud(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libattn_b200.so"))
